@@ -1,0 +1,206 @@
+"""ctypes front for the plain C oracle -- TEST INFRASTRUCTURE, not product code.
+
+Argument marshalling only: every arithmetic step is in ``gpusq_oracle.c``.
+Arrays are numpy, C-contiguous; binary16 tensors travel as ``numpy.float16``.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "gpusq_oracle.c")
+_HDR = os.path.join(_HERE, "gpusq_oracle.h")
+_OUT_DIR = os.path.join(_HERE, "_build")
+_OUT = os.path.join(_OUT_DIR, "libgpusq_oracle.so")
+_lock = threading.Lock()
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle with gcc (no fast-math, no FMA contraction)."""
+    os.makedirs(_OUT_DIR, exist_ok=True)
+    stale = (
+        force
+        or not os.path.exists(_OUT)
+        or os.path.getmtime(_OUT) < max(os.path.getmtime(_SRC), os.path.getmtime(_HDR))
+    )
+    if stale:
+        tmp = _OUT + ".%d.tmp" % os.getpid()
+        cmd = ["gcc", "-std=c99", "-O2", "-ffp-contract=off", "-fno-fast-math", "-fPIC",
+               "-shared", "-Wall", "-Wextra", "-o", tmp, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+        os.replace(tmp, _OUT)
+    return _OUT
+
+
+def _load():
+    global _lib
+    with _lock:
+        if _lib is None:
+            lib = ctypes.CDLL(build())
+            vp, i32, i64, f32 = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_float
+            lib.o_prune24.argtypes = [vp, vp, vp, i32, i32]
+            lib.o_quant_weight.argtypes = [vp, vp, vp, i32, i32]
+            lib.o_compress24.argtypes = [vp, vp, vp, i32, i32]
+            lib.o_decompress24.argtypes = [vp, vp, vp, i32, i32]
+            lib.o_quant_act.argtypes = [vp, vp, vp, i32, i64, i32]
+            lib.o_spgemm_acc.argtypes = [vp, vp, vp, vp, i64, i32, i32]
+            lib.o_spgemm_acc.restype = i64
+            lib.o_spgemm_acc_rows.argtypes = [vp, vp, vp, vp, i64, vp, i32, i32]
+            lib.o_spgemm_acc_rows.restype = i64
+            lib.o_epilogue.argtypes = [vp, vp, f32, vp, i32, i32, f32, vp, i64, i32]
+            lib.o_f32_to_f16.argtypes = [f32]
+            lib.o_f32_to_f16.restype = ctypes.c_uint16
+            lib.o_f16_to_f32.argtypes = [ctypes.c_uint16]
+            lib.o_f16_to_f32.restype = f32
+            lib.o_sqnr_db.argtypes = [vp, vp, i64]
+            lib.o_sqnr_db.restype = ctypes.c_double
+            for name in ("o_prune24", "o_quant_weight", "o_compress24", "o_decompress24",
+                         "o_quant_act", "o_epilogue"):
+                getattr(lib, name).restype = None
+            _lib = lib
+    return _lib
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _c(a, dtype):
+    a = np.ascontiguousarray(a, dtype=dtype)
+    return a
+
+
+def prune24(W, return_mask=False):
+    W = _c(W, np.float32)
+    N, K = W.shape
+    assert K % 4 == 0
+    Wp = np.empty_like(W)
+    mask = np.empty((N, K // 4), np.uint8)
+    _load().o_prune24(_p(W), _p(Wp), _p(mask), N, K)
+    return (Wp, mask) if return_mask else Wp
+
+
+def quant_weight(Wp):
+    Wp = _c(Wp, np.float32)
+    N, K = Wp.shape
+    Wq = np.empty((N, K), np.int8)
+    s = np.empty((N,), np.float32)
+    _load().o_quant_weight(_p(Wp), _p(Wq), _p(s), N, K)
+    return Wq, s
+
+
+def compress24(Wq):
+    Wq = _c(Wq, np.int8)
+    N, K = Wq.shape
+    assert K % 8 == 0
+    vals = np.empty((N, K // 2), np.int8)
+    meta = np.empty((N, K // 8), np.uint8)
+    _load().o_compress24(_p(Wq), _p(vals), _p(meta), N, K)
+    return vals, meta
+
+
+def decompress24(vals, meta):
+    vals = _c(vals, np.int8)
+    meta = _c(meta, np.uint8)
+    N, K = vals.shape[0], vals.shape[1] * 2
+    assert meta.shape == (N, K // 8)
+    Wq = np.empty((N, K), np.int8)
+    _load().o_decompress24(_p(vals), _p(meta), _p(Wq), N, K)
+    return Wq
+
+
+def quant_act(X, x_scale=None):
+    """X float16 [M, K]; x_scale None => computed (mode 0), else supplied (mode 1)."""
+    X = _c(X, np.float16)
+    M, K = X.shape
+    Xq = np.empty((M, K), np.int8)
+    s = np.zeros((1,), np.float32)
+    mode = 0
+    if x_scale is not None:
+        s[0] = x_scale
+        mode = 1
+    _load().o_quant_act(_p(X.view(np.uint16)), _p(Xq), _p(s), mode, M, K)
+    return Xq, np.float32(s[0])
+
+
+def spgemm_acc(Xq, vals, meta):
+    Xq, vals, meta = _c(Xq, np.int8), _c(vals, np.int8), _c(meta, np.uint8)
+    M, K = Xq.shape
+    N = vals.shape[0]
+    assert vals.shape == (N, K // 2) and meta.shape == (N, K // 8)
+    acc = np.empty((M, N), np.int32)
+    ovf = _load().o_spgemm_acc(_p(Xq), _p(vals), _p(meta), _p(acc), M, N, K)
+    assert ovf == 0, "INT32 overflow in %d sums" % ovf
+    return acc
+
+
+def spgemm_acc_rows(Xq, vals, meta, rows):
+    Xq, vals, meta = _c(Xq, np.int8), _c(vals, np.int8), _c(meta, np.uint8)
+    rows = _c(rows, np.int64)
+    M, K = Xq.shape
+    N = vals.shape[0]
+    assert rows.min() >= 0 and rows.max() < M
+    acc = np.empty((rows.size, N), np.int32)
+    ovf = _load().o_spgemm_acc_rows(_p(Xq), _p(vals), _p(meta), _p(rows), rows.size,
+                                    _p(acc), N, K)
+    assert ovf == 0
+    return acc
+
+
+_OUT_DTYPES = {0: np.float16, 1: np.int8, 2: np.int32}
+
+
+def epilogue(acc, w_scale, x_scale, bias=None, act=0, out_type=0, out_scale=1.0):
+    acc = _c(acc, np.int32)
+    w_scale = _c(w_scale, np.float32)
+    if bias is not None:
+        bias = _c(bias, np.float32)
+    N = acc.shape[-1]
+    Y = np.empty(acc.shape, _OUT_DTYPES[out_type])
+    _load().o_epilogue(_p(acc), _p(w_scale), float(x_scale), _p(bias), act, out_type,
+                       float(out_scale), _p(Y), acc.size, N)
+    return Y
+
+
+def f32_to_f16_bits(x: float) -> int:
+    return int(_load().o_f32_to_f16(float(np.float32(x))))
+
+
+def f16_bits_to_f32(h: int) -> float:
+    return float(_load().o_f16_to_f32(int(h)))
+
+
+def sqnr_db(ref, test) -> float:
+    ref, test = _c(ref, np.float32), _c(test, np.float32)
+    return float(_load().o_sqnr_db(_p(ref), _p(test), ref.size))
+
+
+# ---- the two call stacks of the path, as compositions of the steps above ----
+
+def prepare_weight(W):
+    """Offline weight preparation: prune -> quantise -> compress."""
+    Wp, mask = prune24(W, return_mask=True)
+    Wq, w_scale = quant_weight(Wp)
+    vals, meta = compress24(Wq)
+    return {"Wp": Wp, "mask": mask, "Wq": Wq, "w_scale": w_scale, "vals": vals, "meta": meta}
+
+
+def layer_forward(X, prep, bias=None, act=0, out_type=0, out_scale=1.0, x_scale=None,
+                  rows=None):
+    """Per-inference call: quantise activations -> sparse GEMM -> epilogue.
+
+    rows: optional token-row subset (the activation scale still comes from all of X).
+    """
+    Xq, xs = quant_act(X, x_scale)
+    if rows is None:
+        acc = spgemm_acc(Xq, prep["vals"], prep["meta"])
+    else:
+        acc = spgemm_acc_rows(Xq, prep["vals"], prep["meta"], rows)
+    Y = epilogue(acc, prep["w_scale"], xs, bias, act, out_type, out_scale)
+    return {"Xq": Xq, "x_scale": xs, "acc": acc, "Y": Y}
