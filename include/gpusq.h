@@ -1,0 +1,178 @@
+/*
+ * gpusq -- 2:4 fine-grained structured-sparse INT8 linear layers for NVIDIA
+ * B200 (sm_100a).  C ABI of libgpusq.so.
+ *
+ * The layer is Y = X * W^T with
+ *   W [N, K]  weight: the 2:4-sparse operand (matrix A of the paper's Fig. 1)
+ *   X [M, K]  activations: the dense operand (the paper's B, transposed)
+ *   Y [M, N]  output (the paper's C, transposed)
+ * all row-major, densely packed (leading dimension = number of columns).
+ *
+ * Conventions for every call below
+ *   - Every data pointer is a DEVICE pointer owned by the caller.  The library
+ *     allocates nothing, frees nothing and keeps no pointer after the call
+ *     returns (the kernels it enqueued read/write them until the stream
+ *     reaches that point, as with any stream-ordered call).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     Calls enqueue work and return without synchronising.
+ *   - The return value is a gpusq_status.  Argument errors are detected on
+ *     the host before anything is enqueued; no exception, no exit, and no CPU
+ *     fallback: on a device that is not sm_100 the compute calls return
+ *     GPUSQ_ERR_UNSUPPORTED_ARCH.
+ *   - Buffers must not overlap unless a call says it may work in place.
+ *   - Calls are thread-safe when they use distinct streams and distinct
+ *     buffers.
+ */
+#ifndef GPUSQ_H
+#define GPUSQ_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum gpusq_status {
+    GPUSQ_OK = 0,
+    GPUSQ_ERR_NULL = 1,             /* a required pointer is NULL */
+    GPUSQ_ERR_SHAPE = 2,            /* a dimension is <= 0 or violates a divisibility rule */
+    GPUSQ_ERR_ALIGN = 3,            /* a pointer is not aligned as required (16 bytes) */
+    GPUSQ_ERR_WORKSPACE = 4,        /* workspace missing or too small */
+    GPUSQ_ERR_UNSUPPORTED_ARCH = 5, /* current device is not compute capability 10.x */
+    GPUSQ_ERR_CUDA = 6,             /* a CUDA runtime / driver call failed */
+    GPUSQ_ERR_TIMEOUT = 7,          /* a bounded device-side wait expired (see status_buf) */
+    GPUSQ_ERR_ARG = 8               /* an enum argument is out of range */
+} gpusq_status;
+
+enum { GPUSQ_ACT_NONE = 0, GPUSQ_ACT_GELU = 1 };
+enum { GPUSQ_OUT_F16 = 0, GPUSQ_OUT_I8 = 1, GPUSQ_OUT_I32 = 2 };
+enum { GPUSQ_SCALE_COMPUTE = 0, GPUSQ_SCALE_GIVEN = 1 };
+
+/* Human-readable name of a status code (static string, never NULL). */
+const char *gpusq_status_string(int status);
+
+/* ---------------------------------------------------------------------------
+ * gpusq_prune24 -- 2:4 structured pruning along K.
+ * Paper: Sec. 1 and Sec. 3.1 (two of every four contiguous elements on a row
+ * of the sparse matrix are zero); Sec. 3.4 (the dense model is pruned into
+ * the 2:4 sparse one).  Criterion (the paper names none): keep the two
+ * largest magnitudes of each aligned group of four; on equal magnitudes the
+ * lower index is kept; exactly two positions are kept even if they hold
+ * zeros.  NaN inputs give unspecified masks.
+ *   W    [N, K] f32 in.
+ *   Wp   [N, K] f32 out; may be the same pointer as W (in place).
+ *   mask [N, K/4] u8 out, nullable: bit i of the low nibble is set when
+ *        element i of the group is kept.
+ * Requires N > 0, K > 0, K % 4 == 0, W and Wp 16-byte aligned.
+ */
+int gpusq_prune24(const float *W, float *Wp, uint8_t *mask, int N, int K, void *stream);
+
+/* ---------------------------------------------------------------------------
+ * gpusq_quant_weight -- symmetric per-output-channel INT8 weight quantisation.
+ * Paper: Sec. 3.4 (the sparse floating-point model is quantised to INT8 with a
+ * scale factor).  w_scale[n] = max_k |Wp[n,k]| / 127 (1.0 for a zero row);
+ * Wq = clamp(round-half-even(Wp / w_scale[n]), -127, 127); binary32, true
+ * division.
+ *   Wp [N, K] f32 in;  Wq [N, K] i8 out;  w_scale [N] f32 out.
+ * Requires N > 0, K > 0, K % 4 == 0, Wp 16-byte and Wq 4-byte aligned.
+ */
+int gpusq_quant_weight(const float *Wp, int8_t *Wq, float *w_scale, int N, int K, void *stream);
+
+/* ---------------------------------------------------------------------------
+ * gpusq_compress24 -- kept values + 2-bit position metadata.
+ * Paper: Fig. 1, Fig. 2, Sec. 3.1 (M x K/2 values; 2 bits of metadata per kept
+ * value).  Per group of four the kept positions i0 < i1 are derived from the
+ * INT8 codes with the same keep-two rule as gpusq_prune24, so
+ * decompress(compress(Wq)) == Wq for every 2:4 matrix.
+ *   Wq   [N, K]   i8 in.
+ *   vals [N, K/2] i8 out: vals[n, 2g] = Wq[n, 4g+i0], vals[n, 2g+1] = Wq[n, 4g+i1].
+ *   meta [N, K/8] u8 out: nibble = i0 | (i1 << 2); group g of a row is in byte
+ *        g/2, even g in the low nibble.
+ * Requires N > 0, K > 0, K % 8 == 0, Wq 8-byte, vals 4-byte aligned.
+ */
+int gpusq_compress24(const int8_t *Wq, int8_t *vals, uint8_t *meta, int N, int K, void *stream);
+
+/* Inverse of gpusq_compress24 (test and debugging aid). Wq [N, K] i8 out. */
+int gpusq_decompress24(const int8_t *vals, const uint8_t *meta, int8_t *Wq, int N, int K,
+                       void *stream);
+
+/* ---------------------------------------------------------------------------
+ * gpusq_pack24 -- arrange vals + meta the way the sparse tensor-core kernel
+ * reads them (Sec. 3.1: the storage format of the compressed operand; the
+ * layout itself is a hardware detail the paper does not give).
+ * Wpacked holds gpusq_packed_bytes(N, K) bytes, 256-byte aligned:
+ *   [0, Np*Kp/2)            values, row-major [Np, Kp/2], zero padded
+ *   [Np*Kp/2, Np*Kp*5/8)    metadata tiles [Np/128][Kp/128][128 rows][16 bytes]
+ * with Np = N rounded up to 128 and Kp = K rounded up to 128.
+ * Requires N > 0, K > 0, K % 8 == 0.
+ */
+size_t gpusq_packed_bytes(int N, int K);
+int gpusq_pack24(const int8_t *vals, const uint8_t *meta, void *Wpacked, int N, int K,
+                 void *stream);
+
+/* ---------------------------------------------------------------------------
+ * gpusq_quant_act -- symmetric per-tensor INT8 activation quantisation.
+ * Paper: Sec. 2.2 and Sec. 3.4 (a quantise node with one scale factor in front
+ * of each GEMM; the paper learns the factor in training).
+ *   X [M, K] f16 in;  Xq [M, K] i8 out;  x_scale: device float[1].
+ *   scale_mode GPUSQ_SCALE_COMPUTE: *x_scale = max|X| / 127 (1.0 if X is all
+ *     zero) is computed and written; GPUSQ_SCALE_GIVEN: *x_scale is read.
+ *   Xq = clamp(round-half-even(float(X) / *x_scale), -127, 127).
+ *   workspace: device scratch of at least gpusq_quant_act_workspace(M, K)
+ *     bytes, 16-byte aligned, needed for GPUSQ_SCALE_COMPUTE only (may be NULL
+ *     otherwise); its contents on entry do not matter.
+ * Requires M > 0, K > 0, K % 8 == 0, X and Xq 16-byte aligned.
+ */
+size_t gpusq_quant_act_workspace(int64_t M, int K);
+int gpusq_quant_act(const void *X, int8_t *Xq, float *x_scale, int scale_mode, int64_t M, int K,
+                    void *workspace, size_t ws_bytes, void *stream);
+
+/* ---------------------------------------------------------------------------
+ * gpusq_spgemm_i8 -- the fused layer: 2:4-sparse INT8 GEMM + epilogue.
+ * Paper: Fig. 1 and Sec. 3.1 (sparse x dense = dense on the sparse tensor
+ * cores, same result matrix as the dense GEMM); Sec. 2.2 (de-quantise node).
+ *   acc[m,n] = sum_k Wq[n,k] * Xq[m,k]             (INT32, exact)
+ *   y        = fma(float(acc), w_scale[n] * *x_scale, bias ? bias[n] : 0)
+ *   act GPUSQ_ACT_GELU: y = 0.5 * y * erfc(-y / sqrt(2))
+ *   out_type GPUSQ_OUT_F16: Y f16 = round-half-even(y)
+ *            GPUSQ_OUT_I8 : Y i8  = clamp(round-half-even(y / *out_scale), -127, 127)
+ *            GPUSQ_OUT_I32: Y i32 = acc (scales, bias, act ignored)
+ *   Xq [M, K] i8 in;  Wpacked from gpusq_pack24 (N, K);  w_scale [N] f32;
+ *   x_scale device float[1];  bias [N] f32 nullable;  out_scale device
+ *   float[1], GPUSQ_OUT_I8 only;  Y [M, N] out.
+ *   status_buf: device int32[4], nullable.  If given it must be zero on entry;
+ *     a kernel whose bounded wait expires writes {GPUSQ_ERR_TIMEOUT, tile,
+ *     role, stage} there and stops issuing work (the output is then
+ *     undefined).  The host call itself never waits for the device.
+ * Requires M > 0, N % 128 == 0, K % 16 == 0, Xq / Wpacked / Y 16-byte aligned.
+ */
+int gpusq_spgemm_i8(const int8_t *Xq, const void *Wpacked, const float *w_scale,
+                    const float *x_scale, const float *bias, int act, int out_type,
+                    const float *out_scale, void *Y, int64_t M, int N, int K, int32_t *status_buf,
+                    void *stream);
+
+/* ---------------------------------------------------------------------------
+ * gpusq_gemm_i8_dense -- the same kernel and epilogue on the uncompressed
+ * INT8 weight (dense tensor-core instruction): the yardstick for the paper's
+ * "2x math throughput" of the sparse GEMM (Sec. 1, Sec. 3.1).
+ *   Wq [N, K] i8 in (any values; not required to be 2:4).
+ * Other arguments and requirements as gpusq_spgemm_i8.
+ */
+int gpusq_gemm_i8_dense(const int8_t *Xq, const int8_t *Wq, const float *w_scale,
+                        const float *x_scale, const float *bias, int act, int out_type,
+                        const float *out_scale, void *Y, int64_t M, int N, int K,
+                        int32_t *status_buf, void *stream);
+
+/* ---------------------------------------------------------------------------
+ * gpusq_set_block_tokens -- tuning hook for the two GEMM calls (the paper has
+ * no counterpart).  block_t = tokens per output tile, a multiple of 16 in
+ * [16, 240]; 0 restores the automatic choice.  Process-wide; not thread-safe
+ * against concurrent GEMM calls.  Results do not depend on it.
+ */
+int gpusq_set_block_tokens(int block_t);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GPUSQ_H */

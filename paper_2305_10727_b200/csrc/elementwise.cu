@@ -1,0 +1,447 @@
+// HBM-bound operand-preparation kernels of libgpusq: 2:4 pruning, weight and
+// activation quantisation, compression to values + metadata, decompression and
+// packing for the tensor-core kernel.  One pass of coalesced 16-byte accesses
+// per tensor; no shared-memory staging is needed (no reuse across threads).
+#include <cuda_fp16.h>
+
+#include "common.cuh"
+
+namespace gpusq {
+
+constexpr int kThreads = 256;
+
+// ---- keep-two rule (Sec. 1 / Sec. 3.1; criterion: two largest magnitudes, lower index wins ties) ----
+// Element i beats j when mag_i > mag_j, or when they are equal and i < j.  The
+// two elements that win at least two of their three comparisons are kept.
+// Returns the 4-bit keep mask (bit i = element i kept); exactly two bits set.
+template <typename T>
+__device__ __forceinline__ uint32_t keep_two_mask(T m0, T m1, T m2, T m3)
+{
+    const int b01 = m0 >= m1, b02 = m0 >= m2, b03 = m0 >= m3;
+    const int b12 = m1 >= m2, b13 = m1 >= m3, b23 = m2 >= m3;
+    const int w0 = b01 + b02 + b03;
+    const int w1 = (1 - b01) + b12 + b13;
+    const int w2 = (1 - b02) + (1 - b12) + b23;
+    const int w3 = (1 - b03) + (1 - b13) + (1 - b23);
+    return (uint32_t)(w0 >= 2) | ((uint32_t)(w1 >= 2) << 1) | ((uint32_t)(w2 >= 2) << 2) |
+           ((uint32_t)(w3 >= 2) << 3);
+}
+
+// ------------------------------------------------------------------ prune24
+__device__ __forceinline__ float4 prune_group(float4 v, uint32_t &mask)
+{
+    mask = keep_two_mask(fabsf(v.x), fabsf(v.y), fabsf(v.z), fabsf(v.w));
+    v.x = (mask & 1u) ? v.x : 0.0f;
+    v.y = (mask & 2u) ? v.y : 0.0f;
+    v.z = (mask & 4u) ? v.z : 0.0f;
+    v.w = (mask & 8u) ? v.w : 0.0f;
+    return v;
+}
+
+template <int UNROLL>
+__global__ void __launch_bounds__(kThreads)
+prune24_kernel(const float4 *__restrict__ W, float4 *Wp, uint8_t *mask, int64_t groups)
+{
+    // W and Wp may be the same buffer: every thread reads a group before it writes it.
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    for (; i + (UNROLL - 1) * stride < groups; i += UNROLL * stride) {
+        float4 v[UNROLL];
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) v[u] = __ldcs(W + i + u * stride);
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            uint32_t mk;
+            float4 o = prune_group(v[u], mk);
+            __stcs(Wp + i + u * stride, o);
+            if (mask) mask[i + u * stride] = (uint8_t)mk;
+        }
+    }
+    for (; i < groups; i += stride) {
+        uint32_t mk;
+        float4 o = prune_group(__ldcs(W + i), mk);
+        __stcs(Wp + i, o);
+        if (mask) mask[i] = (uint8_t)mk;
+    }
+}
+
+// ------------------------------------------------------------ quantisation
+// code = clamp(round-half-even(x / scale), -127, 127), IEEE division.
+__device__ __forceinline__ int quant_code(float x, float scale)
+{
+    int q = __float2int_rn(__fdiv_rn(x, scale));
+    return max(-127, min(127, q));
+}
+
+__device__ __forceinline__ float scale_from_amax(float amax)
+{
+    return amax == 0.0f ? 1.0f : __fdiv_rn(amax, 127.0f);
+}
+
+__device__ __forceinline__ float block_max(float v, float *red)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    __syncthreads();  // red may still be read from a previous use
+    if (lane == 0) red[warp] = v;
+    __syncthreads();
+    float r = red[0];
+    for (int w = 1; w < (int)(blockDim.x >> 5); ++w) r = fmaxf(r, red[w]);
+    return r;
+}
+
+// One block per output channel (row): pass 1 finds max|w|, pass 2 re-reads the
+// row (L1/L2 resident: a row is at most 20 KB) and writes four codes per store.
+__global__ void __launch_bounds__(kThreads)
+quant_weight_kernel(const float4 *__restrict__ Wp, uint32_t *__restrict__ Wq,
+                    float *__restrict__ w_scale, int N, int K4)
+{
+    __shared__ float red[kThreads / 32];
+    for (int n = blockIdx.x; n < N; n += gridDim.x) {
+        const float4 *row = Wp + (int64_t)n * K4;
+        float m = 0.0f;
+        for (int k = threadIdx.x; k < K4; k += blockDim.x) {
+            float4 v = __ldg(row + k);
+            m = fmaxf(m, fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w))));
+        }
+        const float s = scale_from_amax(block_max(m, red));
+        if (threadIdx.x == 0) w_scale[n] = s;
+        uint32_t *out = Wq + (int64_t)n * K4;
+        for (int k = threadIdx.x; k < K4; k += blockDim.x) {
+            float4 v = __ldg(row + k);
+            uint32_t c = (uint32_t)(quant_code(v.x, s) & 0xFF) | ((uint32_t)(quant_code(v.y, s) & 0xFF) << 8) |
+                         ((uint32_t)(quant_code(v.z, s) & 0xFF) << 16) |
+                         ((uint32_t)(quant_code(v.w, s) & 0xFF) << 24);
+            out[k] = c;
+        }
+    }
+}
+
+// ---------------------------------------------------------------- compress
+// One group = four INT8 codes in a 32-bit word.  Returns the two kept codes
+// (low 16 bits, lower position first) and the metadata nibble i0 | i1 << 2.
+__device__ __forceinline__ void compress_group(uint32_t w, uint32_t &pair, uint32_t &nib)
+{
+    const int c0 = (int8_t)(w & 0xFF), c1 = (int8_t)((w >> 8) & 0xFF);
+    const int c2 = (int8_t)((w >> 16) & 0xFF), c3 = (int8_t)(w >> 24);
+    const uint32_t mk = keep_two_mask(abs(c0), abs(c1), abs(c2), abs(c3));
+    const uint32_t i0 = __ffs(mk) - 1;          // lowest kept position
+    const uint32_t i1 = 31 - __clz(mk);         // highest kept position
+    pair = ((w >> (8 * i0)) & 0xFF) | (((w >> (8 * i1)) & 0xFF) << 8);
+    nib = i0 | (i1 << 2);
+}
+
+// Four groups (16 codes) per thread: 16-byte load, 8-byte + 2-byte stores.  K % 16 == 0.
+__global__ void __launch_bounds__(kThreads)
+compress24_x4_kernel(const uint4 *__restrict__ Wq, uint2 *__restrict__ vals,
+                     uint16_t *__restrict__ meta, int64_t quads)
+{
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < quads; i += stride) {
+        const uint4 w = __ldg(Wq + i);
+        uint32_t p0, p1, p2, p3, n0, n1, n2, n3;
+        compress_group(w.x, p0, n0);
+        compress_group(w.y, p1, n1);
+        compress_group(w.z, p2, n2);
+        compress_group(w.w, p3, n3);
+        vals[i] = make_uint2(p0 | (p1 << 16), p2 | (p3 << 16));
+        meta[i] = (uint16_t)(n0 | (n1 << 4) | (n2 << 8) | (n3 << 12));
+    }
+}
+
+// Two groups per thread for rows whose length is a multiple of 8 only.
+__global__ void __launch_bounds__(kThreads)
+compress24_x2_kernel(const uint2 *__restrict__ Wq, uint32_t *__restrict__ vals,
+                     uint8_t *__restrict__ meta, int64_t pairs)
+{
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < pairs; i += stride) {
+        const uint2 w = __ldg(Wq + i);
+        uint32_t p0, p1, n0, n1;
+        compress_group(w.x, p0, n0);
+        compress_group(w.y, p1, n1);
+        vals[i] = p0 | (p1 << 16);
+        meta[i] = (uint8_t)(n0 | (n1 << 4));
+    }
+}
+
+__device__ __forceinline__ uint32_t decompress_group(uint32_t pair, uint32_t nib)
+{
+    const uint32_t i0 = nib & 3, i1 = (nib >> 2) & 3;
+    uint32_t w = (pair & 0xFF) << (8 * i0);
+    w = (w & ~(0xFFu << (8 * i1))) | (((pair >> 8) & 0xFF) << (8 * i1));
+    return w;
+}
+
+__global__ void __launch_bounds__(kThreads)
+decompress24_kernel(const uint32_t *__restrict__ vals, const uint8_t *__restrict__ meta,
+                    uint2 *__restrict__ Wq, int64_t pairs)
+{
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < pairs; i += stride) {
+        const uint32_t v = __ldg(vals + i);
+        const uint32_t m = __ldg(meta + i);
+        Wq[i] = make_uint2(decompress_group(v & 0xFFFF, m & 0xF), decompress_group(v >> 16, m >> 4));
+    }
+}
+
+// -------------------------------------------------------------------- pack
+// Values: [Np, Kp/2] zero padded.  Metadata: [Np/128][Kp/128][128 rows][16 bytes],
+// i.e. for each 128-row x 128-column block of W the 16 metadata bytes of a row
+// are contiguous and rows follow each other: the 2 KB block is what one
+// tcgen05.cp 128x128b instruction moves into tensor memory.  Padding groups
+// get the well-formed nibble 0x4 (positions 0 and 1); their values are zero.
+__global__ void __launch_bounds__(kThreads)
+pack24_kernel(const int8_t *__restrict__ vals, const uint8_t *__restrict__ meta,
+              uint8_t *__restrict__ packed, int N, int K, int Np, int Kp)
+{
+    const int row_chunks = Kp / 32;                       // 16-byte chunks per padded value row
+    const int64_t val_chunks = (int64_t)Np * row_chunks;
+    const int kt = Kp / 128;
+    const int64_t meta_chunks = (int64_t)Np * kt;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    uint8_t *meta_out = packed + (int64_t)Np * (Kp / 2);
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < val_chunks + meta_chunks;
+         i += stride) {
+        uint32_t w[4];
+        if (i < val_chunks) {
+            const int n = (int)(i / row_chunks), c = (int)(i % row_chunks);
+            const uint32_t *src = reinterpret_cast<const uint32_t *>(vals + (int64_t)n * (K / 2));
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int byte = 16 * c + 4 * j;          // K/2 is a multiple of 4
+                w[j] = (n < N && byte < K / 2) ? __ldg(src + byte / 4) : 0u;
+            }
+            *reinterpret_cast<uint4 *>(packed + i * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+        } else {
+            const int64_t j = i - val_chunks;             // (tile_n, tile_k, r)
+            const int r = (int)(j % 128);
+            const int tk = (int)((j / 128) % kt);
+            const int tn = (int)(j / (128 * (int64_t)kt));
+            const int n = tn * 128 + r;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                uint32_t word = 0;
+#pragma unroll
+                for (int b = 0; b < 4; ++b) {
+                    const int byte = 16 * tk + 4 * q + b;
+                    const uint32_t v = (n < N && byte < K / 8) ? meta[(int64_t)n * (K / 8) + byte] : 0x44u;
+                    word |= v << (8 * b);
+                }
+                w[q] = word;
+            }
+            *reinterpret_cast<uint4 *>(meta_out + j * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+    }
+}
+
+// --------------------------------------------------------------- quant_act
+constexpr int kMaxPartials = 2048;   // workspace: one 32-bit partial maximum per block
+
+__device__ __forceinline__ uint32_t absmax_bits8(uint4 v)
+{
+    // |binary16| as unsigned 15-bit patterns order like the magnitudes (no NaN expected)
+    uint32_t a = __vmaxu2(v.x & 0x7FFF7FFFu, v.y & 0x7FFF7FFFu);
+    uint32_t b = __vmaxu2(v.z & 0x7FFF7FFFu, v.w & 0x7FFF7FFFu);
+    a = __vmaxu2(a, b);
+    return max(a & 0xFFFFu, a >> 16);
+}
+
+__global__ void __launch_bounds__(kThreads)
+act_absmax_kernel(const uint4 *__restrict__ X, uint32_t *__restrict__ partial, int64_t vec8)
+{
+    __shared__ float red[kThreads / 32];
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    uint32_t m = 0;
+    for (; i + 3 * stride < vec8; i += 4 * stride) {
+        uint4 v0 = __ldg(X + i), v1 = __ldg(X + i + stride), v2 = __ldg(X + i + 2 * stride),
+              v3 = __ldg(X + i + 3 * stride);
+        m = max(max(m, absmax_bits8(v0)), max(absmax_bits8(v1), max(absmax_bits8(v2), absmax_bits8(v3))));
+    }
+    for (; i < vec8; i += stride) m = max(m, absmax_bits8(__ldg(X + i)));
+    // binary16 bit patterns below 0x8000 are exact small integers in binary32: reuse the float reduction
+    const float r = block_max((float)m, red);
+    if (threadIdx.x == 0) partial[blockIdx.x] = (uint32_t)r;
+}
+
+__device__ __forceinline__ uint32_t quant4_f16(uint32_t lo, uint32_t hi, float s)
+{
+    const __half2 a = *reinterpret_cast<const __half2 *>(&lo);
+    const __half2 b = *reinterpret_cast<const __half2 *>(&hi);
+    const float2 fa = __half22float2(a), fb = __half22float2(b);
+    return (uint32_t)(quant_code(fa.x, s) & 0xFF) | ((uint32_t)(quant_code(fa.y, s) & 0xFF) << 8) |
+           ((uint32_t)(quant_code(fb.x, s) & 0xFF) << 16) | ((uint32_t)(quant_code(fb.y, s) & 0xFF) << 24);
+}
+
+// n_partials > 0: the scale is derived from the partial maxima and written to
+// *x_scale by block 0; n_partials == 0: *x_scale is read.
+__global__ void __launch_bounds__(kThreads)
+act_quant_kernel(const uint4 *__restrict__ X, uint2 *__restrict__ Xq, float *x_scale,
+                 const uint32_t *__restrict__ partial, int n_partials, int64_t vec8)
+{
+    __shared__ float red[kThreads / 32];
+    float s;
+    if (n_partials > 0) {
+        uint32_t m = 0;
+        for (int i = threadIdx.x; i < n_partials; i += blockDim.x) m = max(m, __ldg(partial + i));
+        const uint32_t bits = (uint32_t)block_max((float)m, red);
+        const float amax = __half2float(__ushort_as_half((unsigned short)bits));
+        s = scale_from_amax(amax);
+        if (blockIdx.x == 0 && threadIdx.x == 0) *x_scale = s;
+    } else {
+        s = *x_scale;
+    }
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    for (; i + stride < vec8; i += 2 * stride) {
+        const uint4 v0 = __ldg(X + i), v1 = __ldg(X + i + stride);
+        __stcs(Xq + i, make_uint2(quant4_f16(v0.x, v0.y, s), quant4_f16(v0.z, v0.w, s)));
+        __stcs(Xq + i + stride, make_uint2(quant4_f16(v1.x, v1.y, s), quant4_f16(v1.z, v1.w, s)));
+    }
+    for (; i < vec8; i += stride) {
+        const uint4 v = __ldg(X + i);
+        __stcs(Xq + i, make_uint2(quant4_f16(v.x, v.y, s), quant4_f16(v.z, v.w, s)));
+    }
+}
+
+inline int grid_for(int64_t items, int per_sm)
+{
+    int64_t blocks = ceil_div(items, kThreads);
+    int64_t cap = (int64_t)num_sms() * per_sm;
+    return (int)(blocks < cap ? (blocks < 1 ? 1 : blocks) : cap);
+}
+
+}  // namespace gpusq
+
+using namespace gpusq;
+
+extern "C" {
+
+int gpusq_prune24(const float *W, float *Wp, uint8_t *mask, int N, int K, void *stream)
+{
+    if (!W || !Wp) return GPUSQ_ERR_NULL;
+    if (N <= 0 || K <= 0 || K % 4) return GPUSQ_ERR_SHAPE;
+    if (!aligned(W, 16) || !aligned(Wp, 16)) return GPUSQ_ERR_ALIGN;
+    if (int st = check_arch()) return st;
+    const int64_t groups = (int64_t)N * (K / 4);
+    prune24_kernel<4><<<grid_for(ceil_div(groups, 4), 8), kThreads, 0, (cudaStream_t)stream>>>(
+        reinterpret_cast<const float4 *>(W), reinterpret_cast<float4 *>(Wp), mask, groups);
+    return launch_status();
+}
+
+int gpusq_quant_weight(const float *Wp, int8_t *Wq, float *w_scale, int N, int K, void *stream)
+{
+    if (!Wp || !Wq || !w_scale) return GPUSQ_ERR_NULL;
+    if (N <= 0 || K <= 0 || K % 4) return GPUSQ_ERR_SHAPE;
+    if (!aligned(Wp, 16) || !aligned(Wq, 4)) return GPUSQ_ERR_ALIGN;
+    if (int st = check_arch()) return st;
+    const int grid = N < num_sms() * 8 ? N : num_sms() * 8;
+    quant_weight_kernel<<<grid, kThreads, 0, (cudaStream_t)stream>>>(
+        reinterpret_cast<const float4 *>(Wp), reinterpret_cast<uint32_t *>(Wq), w_scale, N, K / 4);
+    return launch_status();
+}
+
+int gpusq_compress24(const int8_t *Wq, int8_t *vals, uint8_t *meta, int N, int K, void *stream)
+{
+    if (!Wq || !vals || !meta) return GPUSQ_ERR_NULL;
+    if (N <= 0 || K <= 0 || K % 8) return GPUSQ_ERR_SHAPE;
+    if (!aligned(Wq, 8) || !aligned(vals, 4)) return GPUSQ_ERR_ALIGN;
+    if (int st = check_arch()) return st;
+    const int64_t groups = (int64_t)N * (K / 4);
+    if (K % 16 == 0 && aligned(Wq, 16) && aligned(vals, 8) && aligned(meta, 2)) {
+        compress24_x4_kernel<<<grid_for(groups / 4, 8), kThreads, 0, (cudaStream_t)stream>>>(
+            reinterpret_cast<const uint4 *>(Wq), reinterpret_cast<uint2 *>(vals),
+            reinterpret_cast<uint16_t *>(meta), groups / 4);
+    } else {
+        compress24_x2_kernel<<<grid_for(groups / 2, 8), kThreads, 0, (cudaStream_t)stream>>>(
+            reinterpret_cast<const uint2 *>(Wq), reinterpret_cast<uint32_t *>(vals), meta, groups / 2);
+    }
+    return launch_status();
+}
+
+int gpusq_decompress24(const int8_t *vals, const uint8_t *meta, int8_t *Wq, int N, int K, void *stream)
+{
+    if (!Wq || !vals || !meta) return GPUSQ_ERR_NULL;
+    if (N <= 0 || K <= 0 || K % 8) return GPUSQ_ERR_SHAPE;
+    if (!aligned(Wq, 8) || !aligned(vals, 4)) return GPUSQ_ERR_ALIGN;
+    if (int st = check_arch()) return st;
+    const int64_t pairs = (int64_t)N * (K / 8);
+    decompress24_kernel<<<grid_for(pairs, 8), kThreads, 0, (cudaStream_t)stream>>>(
+        reinterpret_cast<const uint32_t *>(vals), meta, reinterpret_cast<uint2 *>(Wq), pairs);
+    return launch_status();
+}
+
+size_t gpusq_packed_bytes(int N, int K)
+{
+    if (N <= 0 || K <= 0) return 0;
+    const size_t Np = (size_t)round_up(N, 128), Kp = (size_t)round_up(K, 128);
+    return Np * Kp / 2 + Np * Kp / 8;
+}
+
+int gpusq_pack24(const int8_t *vals, const uint8_t *meta, void *Wpacked, int N, int K, void *stream)
+{
+    if (!vals || !meta || !Wpacked) return GPUSQ_ERR_NULL;
+    if (N <= 0 || K <= 0 || K % 8) return GPUSQ_ERR_SHAPE;
+    if (!aligned(vals, 4) || !aligned(Wpacked, 256)) return GPUSQ_ERR_ALIGN;
+    if (int st = check_arch()) return st;
+    const int Np = round_up(N, 128), Kp = round_up(K, 128);
+    const int64_t chunks = (int64_t)Np * (Kp / 32) + (int64_t)Np * (Kp / 128);
+    pack24_kernel<<<grid_for(chunks, 8), kThreads, 0, (cudaStream_t)stream>>>(
+        vals, meta, reinterpret_cast<uint8_t *>(Wpacked), N, K, Np, Kp);
+    return launch_status();
+}
+
+size_t gpusq_quant_act_workspace(int64_t M, int K)
+{
+    (void)M;
+    (void)K;
+    return (size_t)kMaxPartials * sizeof(uint32_t);
+}
+
+int gpusq_quant_act(const void *X, int8_t *Xq, float *x_scale, int scale_mode, int64_t M, int K,
+                    void *workspace, size_t ws_bytes, void *stream)
+{
+    if (!X || !Xq || !x_scale) return GPUSQ_ERR_NULL;
+    if (M <= 0 || K <= 0 || K % 8) return GPUSQ_ERR_SHAPE;
+    if (scale_mode != GPUSQ_SCALE_COMPUTE && scale_mode != GPUSQ_SCALE_GIVEN) return GPUSQ_ERR_ARG;
+    if (!aligned(X, 16) || !aligned(Xq, 16)) return GPUSQ_ERR_ALIGN;
+    if (scale_mode == GPUSQ_SCALE_COMPUTE) {
+        if (!workspace || ws_bytes < gpusq_quant_act_workspace(M, K)) return GPUSQ_ERR_WORKSPACE;
+        if (!aligned(workspace, 16)) return GPUSQ_ERR_ALIGN;
+    }
+    if (int st = check_arch()) return st;
+    const int64_t vec8 = M * (int64_t)K / 8;
+    cudaStream_t s = (cudaStream_t)stream;
+    int n_partials = 0;
+    if (scale_mode == GPUSQ_SCALE_COMPUTE) {
+        n_partials = grid_for(ceil_div(vec8, 4), 8);
+        if (n_partials > kMaxPartials) n_partials = kMaxPartials;
+        act_absmax_kernel<<<n_partials, kThreads, 0, s>>>(reinterpret_cast<const uint4 *>(X),
+                                                         reinterpret_cast<uint32_t *>(workspace), vec8);
+        if (int st = launch_status()) return st;
+    }
+    act_quant_kernel<<<grid_for(ceil_div(vec8, 2), 8), kThreads, 0, s>>>(
+        reinterpret_cast<const uint4 *>(X), reinterpret_cast<uint2 *>(Xq), x_scale,
+        reinterpret_cast<const uint32_t *>(workspace), n_partials, vec8);
+    return launch_status();
+}
+
+const char *gpusq_status_string(int status)
+{
+    switch (status) {
+    case GPUSQ_OK: return "GPUSQ_OK";
+    case GPUSQ_ERR_NULL: return "GPUSQ_ERR_NULL: a required pointer is NULL";
+    case GPUSQ_ERR_SHAPE: return "GPUSQ_ERR_SHAPE: a dimension is not positive or breaks a divisibility rule";
+    case GPUSQ_ERR_ALIGN: return "GPUSQ_ERR_ALIGN: a pointer is not aligned as required";
+    case GPUSQ_ERR_WORKSPACE: return "GPUSQ_ERR_WORKSPACE: workspace missing or too small";
+    case GPUSQ_ERR_UNSUPPORTED_ARCH: return "GPUSQ_ERR_UNSUPPORTED_ARCH: device is not compute capability 10.x";
+    case GPUSQ_ERR_CUDA: return "GPUSQ_ERR_CUDA: a CUDA call failed";
+    case GPUSQ_ERR_TIMEOUT: return "GPUSQ_ERR_TIMEOUT: a bounded device-side wait expired";
+    case GPUSQ_ERR_ARG: return "GPUSQ_ERR_ARG: an enum argument is out of range";
+    default: return "unknown gpusq status";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,457 @@
+// The fused layer kernel of libgpusq: INT8 GEMM on the 5th-generation tensor
+// cores (tcgen05), 2:4-sparse or dense weight operand, INT32 accumulators in
+// tensor memory, and the de-quantise / bias / GELU / convert epilogue.
+//
+// Orientation.  The layer is Y[M,N] = X[M,K] * W[N,K]^T.  tcgen05.mma.sp wants
+// the sparse operand as MMA-A, so the kernel computes Y^T = W * X^T:
+//   MMA-M = 128 output features (one tensor-memory lane each),
+//   MMA-N = block_t tokens (one 32-bit tensor-memory column each),
+//   MMA-K = 64 (sparse) or 32 (dense) per instruction, 128 per pipeline stage.
+//
+// One persistent CTA per SM, six warps:
+//   warp 0    TMA producer (one elected lane): W values, W metadata, X tile
+//   warp 1    tensor-memory owner and MMA issuer (one elected lane)
+//   warps 2-5 epilogue, one per 32-lane quarter of tensor memory
+// Stages are handed over with mbarriers (full/empty per smem stage,
+// full/empty per accumulator buffer); two accumulator buffers let the
+// epilogue of tile i overlap the main loop of tile i+1.
+#include <cuda.h>
+#include <cuda_fp16.h>
+
+#include <mutex>
+
+#include "common.cuh"
+#include "ptx.cuh"
+
+namespace gpusq {
+
+constexpr int kBlockF = 128;        // features per tile
+constexpr int kBlockK = 128;        // K per stage
+constexpr int kMaxBlockT = 240;     // tokens per tile (runtime value, multiple of 16)
+constexpr int kNumThreads = 192;
+constexpr int kTmemCols = 512;
+constexpr int kAccStride = 240;     // column offset of the second accumulator
+constexpr int kMetaCol = 480;       // metadata slots: 4 columns per stage from here
+
+template <bool kSparse>
+struct Cfg {
+    static constexpr int kABytes = kSparse ? kBlockF * 64 : kBlockF * 128;
+    static constexpr int kBBytes = kMaxBlockT * 128;
+    static constexpr int kMetaBytes = kSparse ? 2048 : 0;
+    static constexpr int kStageBytes = kABytes + kBBytes + kMetaBytes;
+    static constexpr int kStages = kSparse ? 5 : 4;
+    static constexpr int kCtlBytes = 1024;
+    static constexpr int kSmemBytes = kStages * kStageBytes + kCtlBytes + 1024 /* alignment slack */;
+    static constexpr int kMmasPerStage = kSparse ? 2 : 4;
+    static constexpr int kAStepBytes = 32;                    // per MMA along K, both variants
+    static constexpr int kBStepBytes = kSparse ? 64 : 32;
+    static constexpr int kASwizzle = kSparse ? 64 : 128;
+};
+
+struct Ctl {
+    uint64_t full[8];
+    uint64_t empty[8];
+    uint64_t tmem_full[2];
+    uint64_t tmem_empty[2];
+    uint64_t drain;
+    uint32_t tmem_base;
+    uint32_t abort_flag;
+};
+
+struct GemmParams {
+    const uint8_t *meta;        // packed metadata tiles (sparse only)
+    const float *w_scale;
+    const float *x_scale;
+    const float *bias;
+    const float *out_scale;
+    void *Y;
+    int32_t *status;
+    int64_t M;
+    int N;
+    int K;
+    int block_t;
+    int act;
+    int out_type;
+};
+
+__device__ __forceinline__ void report_timeout(const GemmParams &p, Ctl *ctl, int tile, int role, int stage)
+{
+    if (atomicExch(&ctl->abort_flag, 1u) == 0u && p.status) {
+        if (atomicCAS(p.status, 0, GPUSQ_ERR_TIMEOUT) == 0) {
+            p.status[1] = tile;
+            p.status[2] = role;
+            p.status[3] = stage;
+        }
+    }
+}
+
+// exact-erf GELU in the erfc form: relative accuracy is kept for negative y
+__device__ __forceinline__ float gelu_erfc(float y)
+{
+    return 0.5f * y * erfcf(-y * 0.70710678118654752440f);
+}
+
+template <bool kSparse>
+__global__ void __launch_bounds__(kNumThreads, 1)
+gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+               const GemmParams p)
+{
+    using C = Cfg<kSparse>;
+    extern __shared__ uint8_t smem_raw[];
+    // operand tiles need 1024-byte alignment for the 128-byte swizzle
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    Ctl *ctl = reinterpret_cast<Ctl *>(smem + C::kStages * C::kStageBytes);
+    volatile uint32_t *abort_flag = &ctl->abort_flag;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int block_t = p.block_t;
+    const int tiles_n = p.N / kBlockF;
+    const int tiles_m = (int)((p.M + block_t - 1) / block_t);
+    const int num_tiles = tiles_n * tiles_m;
+    const int num_kb = (p.K + kBlockK - 1) / kBlockK;
+    const uint32_t stage_tx = (uint32_t)(C::kABytes + block_t * 128 + C::kMetaBytes);
+
+    auto a_smem = [&](int s) { return smem + s * C::kStageBytes; };
+    auto b_smem = [&](int s) { return smem + s * C::kStageBytes + C::kABytes; };
+    auto m_smem = [&](int s) { return smem + s * C::kStageBytes + C::kABytes + C::kBBytes; };
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < C::kStages; ++s) {
+            ptx::mbar_init(ptx::smem_u32(&ctl->full[s]), 1);
+            ptx::mbar_init(ptx::smem_u32(&ctl->empty[s]), 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            ptx::mbar_init(ptx::smem_u32(&ctl->tmem_full[a]), 1);
+            ptx::mbar_init(ptx::smem_u32(&ctl->tmem_empty[a]), 4);
+        }
+        ptx::mbar_init(ptx::smem_u32(&ctl->drain), 1);
+        ctl->abort_flag = 0;
+        ptx::fence_barrier_init();
+        ptx::prefetch_tensormap(&map_a);
+        ptx::prefetch_tensormap(&map_b);
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(ptx::smem_u32(&ctl->tmem_base), kTmemCols);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ producer
+        if (ptx::elect_one()) {
+            int stage = 0;
+            uint32_t phase = 0;
+            uint32_t issued = 0;            // bit s: a load into stage s was issued
+            uint32_t last_parity = 0;       // bit s: parity of the last phase issued into stage s
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+                const int tn = tile % tiles_n, tm = tile / tiles_n;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    bool to;
+                    if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag, to)) {
+                        if (to) report_timeout(p, ctl, tile, 0, stage);
+                        ok = false;
+                        break;
+                    }
+                    const uint32_t bar = ptx::smem_u32(&ctl->full[stage]);
+                    ptx::mbar_arrive_expect_tx(bar, stage_tx);
+                    ptx::tma_load_2d(ptx::smem_u32(a_smem(stage)), &map_a, bar,
+                                     kb * (kSparse ? 64 : 128), tn * kBlockF);
+                    ptx::tma_load_2d(ptx::smem_u32(b_smem(stage)), &map_b, bar, kb * kBlockK, tm * block_t);
+                    if (kSparse) {
+                        const uint8_t *src = p.meta + ((int64_t)tn * num_kb + kb) * 2048;
+                        ptx::bulk_load(ptx::smem_u32(m_smem(stage)), src, 2048, bar);
+                    }
+                    issued |= 1u << stage;
+                    last_parity = (last_parity & ~(1u << stage)) | (phase << stage);
+                    if (++stage == C::kStages) {
+                        stage = 0;
+                        phase ^= 1u;
+                    }
+                }
+            }
+            if (*abort_flag) {
+                // do not leave while bulk copies may still land in this CTA's shared memory
+                for (int s = 0; s < C::kStages; ++s) {
+                    if (issued & (1u << s)) {
+                        uint32_t none = 0;
+                        bool to;
+                        (void)ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->full[s]), (last_parity >> s) & 1u, &none, to);
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------------------------------------------------- MMA issuer
+        if (ptx::elect_one()) {
+            const uint32_t idesc = ptx::make_idesc_i8(kBlockF, block_t, kSparse);
+            int stage = 0;
+            uint32_t phase = 0;
+            int local = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++local) {
+                const int acc = local & 1;
+                const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
+                bool to;
+                if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->tmem_empty[acc]), acc_phase ^ 1u, abort_flag, to)) {
+                    if (to) report_timeout(p, ctl, tile, 1, 100 + acc);
+                    ok = false;
+                    break;
+                }
+                ptx::tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kAccStride);
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->full[stage]), phase, abort_flag, to)) {
+                        if (to) report_timeout(p, ctl, tile, 1, stage);
+                        ok = false;
+                        break;
+                    }
+                    ptx::tc_fence_after();
+                    const uint32_t meta_t = tmem_base + (uint32_t)(kMetaCol + 4 * stage);
+                    if (kSparse) {
+                        ptx::tc_cp_128x128b(meta_t, ptx::make_smem_desc(ptx::smem_u32(m_smem(stage)), 128, 0));
+                    }
+                    const uint64_t adesc = ptx::make_smem_desc(ptx::smem_u32(a_smem(stage)), C::kASwizzle * 8, C::kASwizzle);
+                    const uint64_t bdesc = ptx::make_smem_desc(ptx::smem_u32(b_smem(stage)), 1024, 128);
+#pragma unroll
+                    for (int k = 0; k < C::kMmasPerStage; ++k) {
+                        const uint64_t ad = adesc + (uint64_t)((k * C::kAStepBytes) >> 4);
+                        const uint64_t bd = bdesc + (uint64_t)((k * C::kBStepBytes) >> 4);
+                        const uint32_t accum = (kb | k) != 0 ? 1u : 0u;
+                        if (kSparse)
+                            ptx::tc_mma_sp_i8(d_tmem, ad, bd, meta_t + 2u * k, idesc, accum);
+                        else
+                            ptx::tc_mma_i8(d_tmem, ad, bd, idesc, accum);
+                    }
+                    ptx::tc_commit(ptx::smem_u32(&ctl->empty[stage]));   // stage reusable once these MMAs are done
+                    if (++stage == C::kStages) {
+                        stage = 0;
+                        phase ^= 1u;
+                    }
+                }
+                if (ok) ptx::tc_commit(ptx::smem_u32(&ctl->tmem_full[acc]));
+            }
+            if (*abort_flag) {
+                // let every MMA issued so far retire before tensor memory is released
+                ptx::tc_commit(ptx::smem_u32(&ctl->drain));
+                uint32_t none = 0;
+                bool to;
+                (void)ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->drain), 0, &none, to);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue
+        const int quarter = warp & 3;                      // tensor-memory lanes [32q, 32q+32)
+        const float x_scale = (p.out_type == GPUSQ_OUT_I32) ? 1.0f : __ldg(p.x_scale);
+        const float out_scale = (p.out_type == GPUSQ_OUT_I8) ? __ldg(p.out_scale) : 1.0f;
+        int local = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++local) {
+            const int tn = tile % tiles_n, tm = tile / tiles_n;
+            const int acc = local & 1;
+            const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
+            const int n = tn * kBlockF + quarter * 32 + lane;      // this thread's output feature
+            float sc = 1.0f, bi = 0.0f;
+            if (p.out_type != GPUSQ_OUT_I32) {
+                sc = __fmul_rn(__ldg(p.w_scale + n), x_scale);
+                bi = p.bias ? __ldg(p.bias + n) : 0.0f;
+            }
+            bool to;
+            if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->tmem_full[acc]), acc_phase, abort_flag, to)) {
+                if (to && lane == 0) report_timeout(p, ctl, tile, 2, 100 + acc);
+                ok = false;
+                break;
+            }
+            ptx::tc_fence_after();
+            const int64_t m0 = (int64_t)tm * block_t;
+            for (int c = 0; c < block_t / 16; ++c) {
+                uint32_t r[16];
+                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * kAccStride + c * 16);
+                ptx::tmem_ld_32x32b_x16(taddr, r);
+                ptx::tmem_ld_wait();
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const int64_t m = m0 + c * 16 + j;
+                    if (m < p.M) {
+                        const int32_t a = (int32_t)r[j];
+                        if (p.out_type == GPUSQ_OUT_I32) {
+                            reinterpret_cast<int32_t *>(p.Y)[m * p.N + n] = a;
+                        } else {
+                            float y = __fmaf_rn(__int2float_rn(a), sc, bi);
+                            if (p.act == GPUSQ_ACT_GELU) y = gelu_erfc(y);
+                            if (p.out_type == GPUSQ_OUT_F16) {
+                                reinterpret_cast<__half *>(p.Y)[m * p.N + n] = __float2half_rn(y);
+                            } else {
+                                int q = __float2int_rn(__fdiv_rn(y, out_scale));
+                                q = max(-127, min(127, q));
+                                reinterpret_cast<int8_t *>(p.Y)[m * p.N + n] = (int8_t)q;
+                            }
+                        }
+                    }
+                }
+            }
+            ptx::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctl->tmem_empty[acc]));
+        }
+    }
+
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after();
+        ptx::tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+// ------------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void *f = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(f);
+    });
+    return fn;
+}
+
+// 2-D row-major byte matrix [rows, row_bytes]; box = [box_rows, box_bytes]
+static bool make_map_u8(CUtensorMap *map, const void *base, uint64_t rows, uint64_t row_bytes,
+                        uint32_t box_bytes, uint32_t box_rows, CUtensorMapSwizzle swz)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {row_bytes, rows};
+    cuuint64_t strides[1] = {row_bytes};
+    cuuint32_t box[2] = {box_bytes, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static int g_block_t_override = 0;
+
+// Tokens per tile: a multiple of 16 up to 240 chosen so that the last wave of
+// tiles over the SMs is as full as possible (per-tile cost ~ block_t + fixed part).
+static int choose_block_t(int64_t M, int tiles_n, int sms)
+{
+    if (g_block_t_override) return g_block_t_override;
+    int best = 240;
+    double best_cost = 1e300;
+    for (int bt = 240; bt >= 32; bt -= 16) {
+        const int64_t tiles = (int64_t)tiles_n * ceil_div(M, bt);
+        const int64_t waves = ceil_div(tiles, sms);
+        const double cost = (double)waves * (bt + 48);
+        if (cost < best_cost * 0.999) {
+            best_cost = cost;
+            best = bt;
+        }
+    }
+    return best;
+}
+
+template <bool kSparse>
+static int launch_gemm(const int8_t *Xq, const void *Wsrc, const float *w_scale, const float *x_scale,
+                       const float *bias, int act, int out_type, const float *out_scale, void *Y, int64_t M,
+                       int N, int K, int32_t *status_buf, void *stream)
+{
+    using C = Cfg<kSparse>;
+    if (!Xq || !Wsrc || !Y) return GPUSQ_ERR_NULL;
+    if (out_type < 0 || out_type > 2 || act < 0 || act > 1) return GPUSQ_ERR_ARG;
+    if (out_type != GPUSQ_OUT_I32 && (!w_scale || !x_scale)) return GPUSQ_ERR_NULL;
+    if (out_type == GPUSQ_OUT_I8 && !out_scale) return GPUSQ_ERR_NULL;
+    if (M <= 0 || N <= 0 || K <= 0 || N % kBlockF || K % 16 || M > 0x7FFFFFFF) return GPUSQ_ERR_SHAPE;
+    if (!aligned(Xq, 16) || !aligned(Wsrc, 16) || !aligned(Y, 16)) return GPUSQ_ERR_ALIGN;
+    if (int st = check_arch()) return st;
+
+    const int sms = num_sms();
+    const int tiles_n = N / kBlockF;
+    const int block_t = choose_block_t(M, tiles_n, sms);
+    const int Kp = round_up(K, 128), Np = round_up(N, 128);
+
+    CUtensorMap map_a, map_b;
+    bool ok;
+    if (kSparse)
+        ok = make_map_u8(&map_a, Wsrc, (uint64_t)Np, (uint64_t)Kp / 2, 64, kBlockF, CU_TENSOR_MAP_SWIZZLE_64B);
+    else
+        ok = make_map_u8(&map_a, Wsrc, (uint64_t)N, (uint64_t)K, 128, kBlockF, CU_TENSOR_MAP_SWIZZLE_128B);
+    ok = ok && make_map_u8(&map_b, Xq, (uint64_t)M, (uint64_t)K, 128, (uint32_t)block_t, CU_TENSOR_MAP_SWIZZLE_128B);
+    if (!ok) return GPUSQ_ERR_CUDA;
+
+    GemmParams p;
+    p.meta = kSparse ? reinterpret_cast<const uint8_t *>(Wsrc) + (size_t)Np * (Kp / 2) : nullptr;
+    p.w_scale = w_scale;
+    p.x_scale = x_scale;
+    p.bias = bias;
+    p.out_scale = out_scale;
+    p.Y = Y;
+    p.status = status_buf;
+    p.M = M;
+    p.N = N;
+    p.K = K;
+    p.block_t = block_t;
+    p.act = act;
+    p.out_type = out_type;
+
+    static std::once_flag attr_once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(attr_once, [] {
+        attr_err = cudaFuncSetAttribute(gemm_i8_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        Cfg<true>::kSmemBytes);
+        if (attr_err == cudaSuccess)
+            attr_err = cudaFuncSetAttribute(gemm_i8_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            Cfg<false>::kSmemBytes);
+    });
+    if (attr_err != cudaSuccess) return GPUSQ_ERR_CUDA;
+
+    const int64_t tiles = (int64_t)tiles_n * ceil_div(M, block_t);
+    const int grid = (int)(tiles < sms ? tiles : sms);
+    gemm_i8_kernel<kSparse><<<grid, kNumThreads, C::kSmemBytes, (cudaStream_t)stream>>>(map_a, map_b, p);
+    return launch_status();
+}
+
+}  // namespace gpusq
+
+using namespace gpusq;
+
+extern "C" {
+
+int gpusq_spgemm_i8(const int8_t *Xq, const void *Wpacked, const float *w_scale, const float *x_scale,
+                    const float *bias, int act, int out_type, const float *out_scale, void *Y, int64_t M, int N,
+                    int K, int32_t *status_buf, void *stream)
+{
+    if (Wpacked && !aligned(Wpacked, 256)) return GPUSQ_ERR_ALIGN;
+    return launch_gemm<true>(Xq, Wpacked, w_scale, x_scale, bias, act, out_type, out_scale, Y, M, N, K, status_buf,
+                             stream);
+}
+
+int gpusq_gemm_i8_dense(const int8_t *Xq, const int8_t *Wq, const float *w_scale, const float *x_scale,
+                        const float *bias, int act, int out_type, const float *out_scale, void *Y, int64_t M, int N,
+                        int K, int32_t *status_buf, void *stream)
+{
+    return launch_gemm<false>(Xq, Wq, w_scale, x_scale, bias, act, out_type, out_scale, Y, M, N, K, status_buf,
+                              stream);
+}
+
+int gpusq_set_block_tokens(int block_t)
+{
+    if (block_t != 0 && (block_t < 16 || block_t > kMaxBlockT || block_t % 16)) return GPUSQ_ERR_ARG;
+    g_block_t_override = block_t;
+    return GPUSQ_OK;
+}
+
+}  // extern "C"
