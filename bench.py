@@ -1,0 +1,447 @@
+#!/usr/bin/env python
+"""Benchmark of the 2:4-sparse INT8 linear-layer path on B200.
+
+One step = one per-inference pass of a transformer block's four linear layers
+(QKV, proj, fc1+GELU, fc2) over one batch of synthetic activations: for every
+layer, activation quantisation (FP16 -> INT8, per-tensor absmax scale) followed
+by the fused sparse GEMM + de-quantise/bias/GELU epilogue writing FP16.  The
+offline weight preparation (prune -> quantise -> compress -> pack) runs once
+before the timed region and is reported separately under "prep".
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle on the
+host cores instead (a deliberately plain program: context, not a target).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2305_10727_b200 import inputs  # noqa: E402
+
+METRIC = "sparse INT8 GEMM effective TOPS (dense-equivalent 2*M*N*K / time), ViT-B block linears at batch 64"
+UNIT = "TOPS"
+NOMINAL_SPARSE_INT8_TOPS = 9000.0      # NVIDIA's dense-half figure for B200 INT8 with 2:4 sparsity (4 x 2250 BF16)
+NOMINAL_BF16_TFLOPS = 2250.0
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# DRAM bytes per launch of the dominant kernel from the ncu capture summarised in
+# profiles/gemm_i8_sparse_deit_base_qkv.md (None until a capture exists)
+NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        p["_source"] = "measured"
+        return p
+    p = dict(FALLBACK_PEAKS)
+    p["_source"] = "fallback"
+    return p
+
+
+def layer_flops(M, L):
+    return 2.0 * M * L.N * L.K
+
+
+def layer_bytes(M, L):
+    # algorithmic bytes of the fused GEMM: INT8 activations in, compressed weight (0.625 B/param)
+    # plus scale and bias vectors in, FP16 out
+    return M * L.K + 0.625 * L.N * L.K + 8 * L.N + 2.0 * M * L.N
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.tmp = None
+
+    def start(self):
+        try:
+            self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu_index), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "50"], stdout=self.tmp, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        time.sleep(0.12)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.tmp.flush()
+        self.tmp.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.tmp.read().splitlines():
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        self.tmp.close()
+        try:
+            os.unlink(self.tmp.name)
+        except OSError:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# --------------------------------------------------------------------------- reference arm
+def run_reference(args, cfg):
+    """The CPU oracle, as it stands, on a bounded sample of the same workload.
+
+    Each step runs the block's four layers on the first `rows` token rows; rows is sized from a
+    short calibration so that the whole --steps/--warmup run stays near a minute of CPU work.
+    """
+    import oracle
+    oracle.build()
+    layers = cfg.layers
+
+    def make(rows):
+        data = []
+        for li, L in enumerate(layers):
+            d = inputs.make_layer_inputs(cfg, li, M=rows)
+            data.append((L, d, oracle.prepare_weight(d["W"])))
+        return data
+
+    def step(data):
+        for L, d, prep in data:
+            oracle.layer_forward(d["X"], prep, d["bias"], act=1 if L.gelu else 0)
+
+    rows = args.ref_rows
+    if rows <= 0:
+        cal = make(16)
+        t0 = time.perf_counter()
+        step(cal)
+        per_row = (time.perf_counter() - t0) / 16
+        budget_s = 60.0
+        rows = int(budget_s / max(per_row, 1e-9) / (args.steps + args.warmup))
+        rows = max(4, min(rows, 512, cfg.M))
+    data = make(rows)
+    flops = sum(layer_flops(rows, L) for L in layers)
+    for _ in range(args.warmup):
+        step(data)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step(data)
+    dt = (time.perf_counter() - t0) / args.steps
+    value = flops / dt / 1e12
+    sample = "first %d token rows of each of the %d layers (of M=%d) per step" % (rows, len(layers), cfg.M)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3 * (cfg.M / rows),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+        "config": {"workload": cfg.name, "M": cfg.M, "layers": [[L.name, L.K, L.N] for L in layers],
+                   "note": "ms_per_step is the sampled step scaled to all M rows"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------------- GPU arm
+def run_gpusq(args, cfg):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2305_10727_b200 import binding as B
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: libgpusq has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    B.load()
+    peaks = load_peaks()
+    M = cfg.M
+    layers = cfg.layers
+
+    # ---- inputs (seeded, synthetic) and offline weight preparation on the device
+    host = [inputs.make_layer_inputs(cfg, li, seed=rank) for li in range(len(layers))]
+    state = []
+    prep_us = {}
+    for li, L in enumerate(layers):
+        h = host[li]
+        W = torch.from_numpy(h["W"]).to(dev)
+        X = torch.from_numpy(h["X"]).to(dev)
+        bias = torch.from_numpy(h["bias"]).to(dev)
+        Wp = torch.empty_like(W)
+        Wq = torch.empty((L.N, L.K), dtype=torch.int8, device=dev)
+        ws = torch.empty((L.N,), dtype=torch.float32, device=dev)
+        vals = torch.empty((L.N, L.K // 2), dtype=torch.int8, device=dev)
+        meta = torch.empty((L.N, L.K // 8), dtype=torch.uint8, device=dev)
+        Wpk = torch.empty((B.packed_bytes(L.N, L.K),), dtype=torch.uint8, device=dev)
+
+        def prep_once():
+            B.prune24(W, Wp=Wp)
+            B.quant_weight(Wp, Wq=Wq, w_scale=ws)
+            B.compress24(Wq, vals=vals, meta=meta)
+            B.pack24(vals, meta, Wpacked=Wpk)
+
+        prep_once()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(5):
+            prep_once()
+        e1.record()
+        torch.cuda.synchronize()
+        prep_us[L.name] = e0.elapsed_time(e1) * 1e3 / 5
+        state.append(dict(L=L, X=X, bias=bias, Wq=Wq, ws=ws, Wpk=Wpk,
+                          Xq=torch.empty((M, L.K), dtype=torch.int8, device=dev),
+                          xs=torch.empty((1,), dtype=torch.float32, device=dev),
+                          wsb=torch.empty((B.quant_act_workspace(M, L.K),), dtype=torch.uint8, device=dev),
+                          Y=torch.empty((M, L.N), dtype=torch.float16, device=dev)))
+    status = torch.zeros(4, dtype=torch.int32, device=dev)
+
+    def layer_quant(s):
+        B.quant_act(s["X"], Xq=s["Xq"], x_scale=s["xs"], workspace=s["wsb"])
+
+    def layer_gemm(s):
+        B.spgemm_i8(s["Xq"], s["Wpk"], s["L"].N, s["ws"], s["xs"], s["bias"],
+                    act=B.ACT_GELU if s["L"].gelu else B.ACT_NONE, out_type=B.OUT_F16, Y=s["Y"], status_buf=status)
+
+    def layer_gemm_dense(s):
+        B.gemm_i8_dense(s["Xq"], s["Wq"], s["ws"], s["xs"], s["bias"],
+                        act=B.ACT_GELU if s["L"].gelu else B.ACT_NONE, out_type=B.OUT_F16, Y=s["Y"],
+                        status_buf=status)
+
+    def step():
+        for s in state:
+            layer_quant(s)
+            layer_gemm(s)
+
+    launches_per_step = 3 * len(state)        # absmax + quantise + GEMM per layer
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    stream = torch.cuda.Stream()
+    torch.cuda.set_stream(stream)
+    graph = None
+    if args.launch == "graph":
+        for _ in range(2):
+            step()
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            step()
+        run_step = graph.replay
+    else:
+        run_step = step
+
+    # ---- headline: K whole steps, inputs resident in HBM
+    for _ in range(max(args.warmup, 3)):
+        run_step()
+    sampler = ClockSampler(local_rank)
+    barrier()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        run_step()
+    e1.record(stream)
+    barrier()
+    ms_step = e0.elapsed_time(e1) / args.steps
+
+    # ---- per-kernel durations over the same K steps, launched eagerly with events on the launch stream
+    def timed_kernel_pass(fn_quant, fn_gemm):
+        evs = []
+        for _ in range(args.steps):
+            for s in state:
+                a, b, c = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+                a.record(stream)
+                fn_quant(s)
+                b.record(stream)
+                fn_gemm(s)
+                c.record(stream)
+                evs.append((s["L"].name, a, b, c))
+        torch.cuda.synchronize()
+        q, g = {}, {}
+        for name, a, b, c in evs:
+            q.setdefault(name, []).append(a.elapsed_time(b) * 1e3)
+            g.setdefault(name, []).append(b.elapsed_time(c) * 1e3)
+        return q, g
+
+    quant_us, gemm_us = timed_kernel_pass(layer_quant, layer_gemm)
+    clocks = sampler.stop()
+    _, dense_us = timed_kernel_pass(lambda s: None, layer_gemm_dense)
+    status_host = status.cpu().tolist()
+
+    if world > 1:
+        t = torch.tensor([ms_step], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_step = float(t.item())
+
+    flops_step = sum(layer_flops(M, L) for L in layers)
+    value = world * flops_step / (ms_step * 1e-3) / 1e12
+
+    # ---- roofline of the dominant kernel (the sparse GEMM, all four shapes of the block)
+    gemm_mean = {k: statistics.fmean(v) for k, v in gemm_us.items()}
+    gemm_total_us = sum(gemm_mean.values())
+    achieved = flops_step / (gemm_total_us * 1e-6) / 1e12
+    sparse_ratio = NOMINAL_SPARSE_INT8_TOPS / NOMINAL_BF16_TFLOPS
+    peak = peaks["bf16_tflops_sustained"] * sparse_ratio
+    bytes_step = sum(layer_bytes(M, L) for L in layers)
+    hbm_achieved = bytes_step / (gemm_total_us * 1e-6) / 1e9
+    per_layer = {}
+    for L in layers:
+        us = gemm_mean[L.name]
+        per_layer[L.name] = {
+            "K": L.K, "N": L.N, "us": round(us, 2), "us_best": round(min(gemm_us[L.name]), 2),
+            "tops": round(layer_flops(M, L) / us / 1e6, 1),
+            "frac_nominal_sparse_peak": round(layer_flops(M, L) / us / 1e6 / NOMINAL_SPARSE_INT8_TOPS, 4),
+            "hbm_gbs": round(layer_bytes(M, L) / us / 1e3, 1),
+            "dense_variant_us": round(statistics.fmean(dense_us[L.name]), 2),
+            "speedup_vs_dense_variant": round(statistics.fmean(dense_us[L.name]) / us, 3),
+            "quant_act_us": round(statistics.fmean(quant_us[L.name]), 2),
+        }
+    roofline = {
+        "bound": "tensor", "kernel": "gemm_i8_kernel<sparse>", "achieved": round(achieved, 1),
+        "peak": round(peak, 1), "unit": "TFLOP/s", "frac": round(achieved / peak, 4), "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH,
+        "peak_source": "%s BF16 sustained x %.0f (nominal INT8-sparse : BF16 ratio)" % (peaks["_source"], sparse_ratio),
+        "frac_of_nominal_9000": round(achieved / NOMINAL_SPARSE_INT8_TOPS, 4),
+        "frac_of_burst_peak": round(achieved / (peaks["bf16_tflops"] * sparse_ratio), 4),
+        "hbm_achieved_gbs": round(hbm_achieved, 1), "hbm_peak_gbs": peaks["hbm_gbs"],
+        "hbm_frac": round(hbm_achieved / peaks["hbm_gbs"], 4),
+        "gemm_block_us": round(gemm_total_us, 2),
+        "timing": "CUDA events on the launch stream around each GEMM launch, eager pass of the same %d steps" % args.steps,
+    }
+
+    # ---- end to end through the public API with host buffers (pinned), copies inside the timed region
+    e2e = None
+    if not args.no_e2e:
+        hX = [torch.from_numpy(h["X"]).pin_memory() for h in host]
+        hY = [torch.empty((M, L.N), dtype=torch.float16).pin_memory() for L in layers]
+        h2d = sum(x.numel() * 2 for x in hX)
+        d2h = sum(y.numel() * 2 for y in hY)
+
+        def e2e_step():
+            for s, hx in zip(state, hX):
+                s["X"].copy_(hx, non_blocking=True)
+            run_step()
+            for s, hy in zip(state, hY):
+                hy.copy_(s["Y"], non_blocking=True)
+
+        for _ in range(3):
+            e2e_step()
+        barrier()
+        n_e2e = max(3, min(args.steps, 10))
+        e0.record(stream)
+        for _ in range(n_e2e):
+            e2e_step()
+        e1.record(stream)
+        barrier()
+        ms_e2e = e0.elapsed_time(e1) / n_e2e
+        if world > 1:
+            t = torch.tensor([ms_e2e], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms_e2e = float(t.item())
+        e2e = {"value": round(world * flops_step / (ms_e2e * 1e-3) / 1e12, 2), "unit": UNIT,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": round(ms_e2e, 4), "steps": n_e2e}
+
+    # ---- CPU baseline: the oracle on a bounded sample (rank 0, N = 1 only)
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        rows = args.ref_rows
+        t_cpu = 0.0
+        for li, L in enumerate(layers):
+            h = host[li]
+            prep = oracle.prepare_weight(h["W"])
+            Xs = np.ascontiguousarray(h["X"][:rows])
+            t0 = time.perf_counter()
+            oracle.layer_forward(Xs, prep, h["bias"], act=1 if L.gelu else 0)
+            t_cpu += time.perf_counter() - t0
+        cpu_tops = sum(layer_flops(rows, L) for L in layers) / t_cpu / 1e12
+        cpu_baseline = {"value": cpu_tops, "unit": UNIT, "cores": 1, "kind": "oracle",
+                        "sample": "first %d of %d token rows of each layer (quantise + GEMM + epilogue), %.1f s"
+                                  % (rows, M, t_cpu)}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": round(ms_step, 5), "block_us": round(ms_step * 1e3, 2),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+            "config": {"workload": cfg.name, "M": M, "layers": [[L.name, L.K, L.N] for L in layers],
+                       "step": "per layer: quant_act (absmax + quantise) + sparse GEMM with fused epilogue, FP16 out",
+                       "launch": args.launch, "l2": "inputs exceed L2: a step touches %.0f MB" % ((bytes_step + sum(2.0 * M * L.K for L in layers)) / 1e6),
+                       "parallelism": "replicas, tokens sharded, no collective" if world > 1 else "single GPU"},
+            "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e,
+            "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
+            "layers": per_layer, "prep_us": {k: round(v, 2) for k, v in prep_us.items()},
+            "device_status": status_host, "peaks": {k: v for k, v in peaks.items() if k in ("hbm_gbs", "bf16_tflops", "bf16_tflops_sustained", "_source")},
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="gpusq", choices=["gpusq", "reference"])
+    ap.add_argument("--config", default="deit_base_b64", choices=inputs.config_names())
+    ap.add_argument("--launch", default="graph", choices=["graph", "eager"])
+    ap.add_argument("--ref-rows", type=int, default=256, help="token rows per layer the CPU oracle is timed on")
+    ap.add_argument("--ref-rows-reference", type=int, default=0,
+                    help="token rows per step for --impl reference (0 = size from a calibration run)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    cfg = inputs.CONFIGS[args.config]
+    if args.impl == "reference":
+        if int(os.environ.get("RANK", "0")) != 0:
+            return
+        args.ref_rows = args.ref_rows_reference
+        run_reference(args, cfg)
+    else:
+        run_gpusq(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,111 @@
+"""GPU parity at the full benchmark sizes, in the launch configuration bench.py
+times (automatic tile choice, persistent grid): the five workload configs,
+every layer.  Weight-side stages and the activation codes are compared with the
+oracle in full; the GEMM and the epilogue are compared on sampled token rows the
+oracle computes one by one (first tile, the ragged last tile, random rows), plus
+an exact column-sum identity that covers every output element, plus equality
+with the dense-instruction variant of the same kernel."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2305_10727_b200 import inputs
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+F16_ULP_TOL = 1
+
+
+@pytest.fixture(scope="module")
+def B():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2305_10727_b200 import binding
+    binding.load()
+    binding.set_block_tokens(0)
+    return binding
+
+
+def cu(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def f16_ulp_distance(a, b):
+    def key(h):
+        u = h.view(np.uint16).astype(np.int32)
+        return np.where(u & 0x8000, -(u & 0x7FFF), u & 0x7FFF)
+    return np.abs(key(np.ascontiguousarray(a)) - key(np.ascontiguousarray(b)))
+
+
+def sample_rows(M, seed, n_random=24):
+    rng = np.random.default_rng(seed)
+    fixed = [0, 1, 15, 16, 127, 128, 239, 240, 255, 256, M - 1, M - 2, M - 17, M // 2]
+    rows = [r for r in fixed if 0 <= r < M] + rng.integers(0, M, n_random).tolist()
+    return np.unique(np.array(rows, np.int64))
+
+
+CASES = [(name, li) for name, cfg in inputs.CONFIGS.items() for li in range(len(cfg.layers))]
+
+
+@pytest.mark.parametrize("name,li", CASES, ids=["%s-%s" % (n, inputs.CONFIGS[n].layers[i].name) for n, i in CASES])
+def test_config_layer(B, name, li):
+    cfg = inputs.CONFIGS[name]
+    L = cfg.layers[li]
+    d = inputs.make_layer_inputs(cfg, li)
+    M = cfg.M
+
+    # ---- offline weight preparation, full comparison
+    prep = oracle.prepare_weight(d["W"])
+    Wp, mask = B.prune24(cu(d["W"]), want_mask=True)
+    Wq, ws = B.quant_weight(Wp)
+    vals, meta = B.compress24(Wq)
+    Wpk = B.pack24(vals, meta)
+    assert np.array_equal(mask.cpu().numpy(), prep["mask"])
+    assert np.array_equal(Wq.cpu().numpy(), prep["Wq"])
+    assert np.array_equal(ws.cpu().numpy(), prep["w_scale"])
+    assert np.array_equal(vals.cpu().numpy(), prep["vals"])
+    assert np.array_equal(meta.cpu().numpy(), prep["meta"])
+
+    # ---- activation quantisation, full comparison
+    Xq_o, xs_o = oracle.quant_act(d["X"])
+    Xq, xs = B.quant_act(cu(d["X"]))
+    assert xs.cpu().numpy()[0] == xs_o
+    assert np.array_equal(Xq.cpu().numpy(), Xq_o)
+
+    # ---- GEMM accumulators
+    status = torch.zeros(4, dtype=torch.int32, device="cuda")
+    acc = B.spgemm_i8(Xq, Wpk, L.N, out_type=B.OUT_I32, status_buf=status)
+    acc_dense = B.gemm_i8_dense(Xq, Wq, out_type=B.OUT_I32, status_buf=status)
+    assert status.cpu().tolist() == [0, 0, 0, 0]
+    assert torch.equal(acc, acc_dense)                   # same C as the dense GEMM, every element
+    rows = sample_rows(M, cfg.cid * 10 + li)
+    acc_rows_o = oracle.spgemm_acc_rows(Xq_o, prep["vals"], prep["meta"], rows)
+    assert np.array_equal(acc[cu(rows)].cpu().numpy(), acc_rows_o)
+    # sum_m acc[m, n] = sum_k Wq[n, k] * (sum_m Xq[m, k]): exact in int64, touches every element
+    col = acc.sum(dim=0, dtype=torch.int64).cpu().numpy()
+    want = prep["Wq"].astype(np.int64) @ Xq_o.astype(np.int64).sum(0)
+    assert np.array_equal(col, want)
+    del acc_dense
+
+    # ---- epilogue, FP16 output
+    act = 1 if L.gelu else 0
+    bias = cu(d["bias"])
+    Y = B.spgemm_i8(Xq, Wpk, L.N, ws, xs, bias, act=act, out_type=B.OUT_F16, status_buf=status)
+    Y_rows_o = oracle.epilogue(acc_rows_o, prep["w_scale"], xs_o, d["bias"], act=act, out_type=0)
+    dist = f16_ulp_distance(Y[cu(rows)].cpu().numpy(), Y_rows_o)
+    assert dist.max() <= F16_ULP_TOL
+    if act == 0:
+        assert dist.max() == 0
+    assert torch.isfinite(Y).all()
+
+    # ---- epilogue, requantised INT8 output (the chained-layer variant)
+    if cfg.int8_out:
+        out_scale = np.float32(float(Y.abs().max().cpu()) / 127.0)
+        Q = B.spgemm_i8(Xq, Wpk, L.N, ws, xs, bias, act=act, out_type=B.OUT_I8,
+                        out_scale=cu(np.array([out_scale], np.float32)), status_buf=status)
+        Q_rows_o = oracle.epilogue(acc_rows_o, prep["w_scale"], xs_o, d["bias"], act=act, out_type=1,
+                                   out_scale=out_scale)
+        diff = np.abs(Q[cu(rows)].cpu().numpy().astype(np.int32) - Q_rows_o.astype(np.int32))
+        assert diff.max() <= (1 if act else 0)
+    assert status.cpu().tolist() == [0, 0, 0, 0]
