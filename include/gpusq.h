@@ -166,8 +166,8 @@ int gpusq_gemm_i8_dense(const int8_t *Xq, const int8_t *Wq, const float *w_scale
 
 /* ---------------------------------------------------------------------------
  * gpusq_set_block_tokens -- tuning hook for the two GEMM calls (the paper has
- * no counterpart).  block_t = tokens per output tile, a multiple of 16 in
- * [16, 240]; 0 restores the automatic choice.  Process-wide; not thread-safe
+ * no counterpart).  block_t = tokens per output tile, a multiple of 32 in
+ * [32, 224]; 0 restores the automatic choice.  Process-wide; not thread-safe
  * against concurrent GEMM calls.  Results do not depend on it.
  */
 int gpusq_set_block_tokens(int block_t);

@@ -8,13 +8,19 @@
 //   MMA-N = block_t tokens (one 32-bit tensor-memory column each),
 //   MMA-K = 64 (sparse) or 32 (dense) per instruction, 128 per pipeline stage.
 //
-// One persistent CTA per SM, six warps:
+// One persistent CTA per SM, ten warps:
 //   warp 0    TMA producer (one elected lane): W values, W metadata, X tile
 //   warp 1    tensor-memory owner and MMA issuer (one elected lane)
-//   warps 2-5 epilogue, one per 32-lane quarter of tensor memory
+//   warps 2-9 epilogue: two warps per 32-lane quarter of tensor memory, which
+//             take alternate 32-token chunks of the tile
 // Stages are handed over with mbarriers (full/empty per smem stage,
 // full/empty per accumulator buffer); two accumulator buffers let the
 // epilogue of tile i overlap the main loop of tile i+1.
+//
+// FP16 epilogue: tcgen05.ld in the 16x256b (accumulator-fragment) shape, FP32
+// math, pack pairs of tokens to f16x2, stmatrix.trans into a 64-byte-swizzled
+// [32 tokens][32 features] staging tile per warp, TMA store to Y (full 64-byte
+// row segments, rows beyond M clipped by the tensor map).
 #include <cuda.h>
 #include <cuda_fp16.h>
 
@@ -27,11 +33,15 @@ namespace gpusq {
 
 constexpr int kBlockF = 128;        // features per tile
 constexpr int kBlockK = 128;        // K per stage
-constexpr int kMaxBlockT = 240;     // tokens per tile (runtime value, multiple of 16)
-constexpr int kNumThreads = 192;
+constexpr int kMaxBlockT = 224;     // tokens per tile (runtime value, multiple of 32)
+constexpr int kChunkT = 32;         // tokens per epilogue chunk
+constexpr int kEpiWarps = 8;
+constexpr int kNumThreads = 64 + 32 * kEpiWarps;
 constexpr int kTmemCols = 512;
-constexpr int kAccStride = 240;     // column offset of the second accumulator
-constexpr int kMetaCol = 480;       // metadata slots: 4 columns per stage from here
+constexpr int kAccStride = 224;     // column offset of the second accumulator
+constexpr int kMetaCol = 448;       // metadata slots: 4 columns per stage from here
+constexpr int kEpiStageBytes = kChunkT * 64;          // [32 tokens][32 features] f16
+constexpr int kEpiBytes = kEpiWarps * 2 * kEpiStageBytes;
 
 template <bool kSparse>
 struct Cfg {
@@ -41,7 +51,7 @@ struct Cfg {
     static constexpr int kStageBytes = kABytes + kBBytes + kMetaBytes;
     static constexpr int kStages = kSparse ? 5 : 4;
     static constexpr int kCtlBytes = 1024;
-    static constexpr int kSmemBytes = kStages * kStageBytes + kCtlBytes + 1024 /* alignment slack */;
+    static constexpr int kSmemBytes = kStages * kStageBytes + kEpiBytes + kCtlBytes + 1024 /* alignment slack */;
     static constexpr int kMmasPerStage = kSparse ? 2 : 4;
     static constexpr int kAStepBytes = 32;                    // per MMA along K, both variants
     static constexpr int kBStepBytes = kSparse ? 64 : 32;
@@ -94,13 +104,14 @@ __device__ __forceinline__ float gelu_erfc(float y)
 template <bool kSparse>
 __global__ void __launch_bounds__(kNumThreads, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-               const GemmParams p)
+               const __grid_constant__ CUtensorMap map_y, const GemmParams p)
 {
     using C = Cfg<kSparse>;
     extern __shared__ uint8_t smem_raw[];
     // operand tiles need 1024-byte alignment for the 128-byte swizzle
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    Ctl *ctl = reinterpret_cast<Ctl *>(smem + C::kStages * C::kStageBytes);
+    uint8_t *epi_smem = smem + C::kStages * C::kStageBytes;
+    Ctl *ctl = reinterpret_cast<Ctl *>(epi_smem + kEpiBytes);
     volatile uint32_t *abort_flag = &ctl->abort_flag;
 
     const int warp = threadIdx.x >> 5;
@@ -123,13 +134,14 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
         for (int a = 0; a < 2; ++a) {
             ptx::mbar_init(ptx::smem_u32(&ctl->tmem_full[a]), 1);
-            ptx::mbar_init(ptx::smem_u32(&ctl->tmem_empty[a]), 4);
+            ptx::mbar_init(ptx::smem_u32(&ctl->tmem_empty[a]), kEpiWarps);
         }
         ptx::mbar_init(ptx::smem_u32(&ctl->drain), 1);
         ctl->abort_flag = 0;
         ptx::fence_barrier_init();
         ptx::prefetch_tensormap(&map_a);
         ptx::prefetch_tensormap(&map_b);
+        if (p.out_type == GPUSQ_OUT_F16) ptx::prefetch_tensormap(&map_y);
     }
     if (warp == 1) {
         ptx::tmem_alloc(ptx::smem_u32(&ctl->tmem_base), kTmemCols);
@@ -246,46 +258,108 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     } else {
         // ------------------------------------------------------------ epilogue
         const int quarter = warp & 3;                      // tensor-memory lanes [32q, 32q+32)
+        const int parity = (warp - 2) >> 2;                // this warp takes chunks parity, parity+2, ...
         const float x_scale = (p.out_type == GPUSQ_OUT_I32) ? 1.0f : __ldg(p.x_scale);
         const float out_scale = (p.out_type == GPUSQ_OUT_I8) ? __ldg(p.out_scale) : 1.0f;
+        const uint32_t stage0 = ptx::smem_u32(epi_smem + (warp - 2) * 2 * kEpiStageBytes);
+        const int chunks = block_t / kChunkT;
+        uint32_t buf = 0;
         int local = 0;
         bool ok = true;
         for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++local) {
             const int tn = tile % tiles_n, tm = tile / tiles_n;
             const int acc = local & 1;
             const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
-            const int n = tn * kBlockF + quarter * 32 + lane;      // this thread's output feature
-            float sc = 1.0f, bi = 0.0f;
-            if (p.out_type != GPUSQ_OUT_I32) {
-                sc = __fmul_rn(__ldg(p.w_scale + n), x_scale);
-                bi = p.bias ? __ldg(p.bias + n) : 0.0f;
-            }
-            bool to;
-            if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->tmem_full[acc]), acc_phase, abort_flag, to)) {
-                if (to && lane == 0) report_timeout(p, ctl, tile, 2, 100 + acc);
-                ok = false;
-                break;
-            }
-            ptx::tc_fence_after();
             const int64_t m0 = (int64_t)tm * block_t;
-            for (int c = 0; c < block_t / 16; ++c) {
-                uint32_t r[16];
-                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * kAccStride + c * 16);
-                ptx::tmem_ld_32x32b_x16(taddr, r);
-                ptx::tmem_ld_wait();
+            const uint32_t tbase = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * kAccStride);
+            bool to;
+            if (p.out_type == GPUSQ_OUT_F16) {
+                // features of this thread: 32q + 16h + 8j + lane/4 (h = lane half of the quarter, j = fragment row)
+                float sc[2][2], bi[2][2];
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const int64_t m = m0 + c * 16 + j;
-                    if (m < p.M) {
-                        const int32_t a = (int32_t)r[j];
-                        if (p.out_type == GPUSQ_OUT_I32) {
-                            reinterpret_cast<int32_t *>(p.Y)[m * p.N + n] = a;
-                        } else {
-                            float y = __fmaf_rn(__int2float_rn(a), sc, bi);
-                            if (p.act == GPUSQ_ACT_GELU) y = gelu_erfc(y);
-                            if (p.out_type == GPUSQ_OUT_F16) {
-                                reinterpret_cast<__half *>(p.Y)[m * p.N + n] = __float2half_rn(y);
+                for (int h = 0; h < 2; ++h)
+#pragma unroll
+                    for (int j = 0; j < 2; ++j) {
+                        const int n = tn * kBlockF + quarter * 32 + 16 * h + 8 * j + (lane >> 2);
+                        sc[h][j] = __fmul_rn(__ldg(p.w_scale + n), x_scale);
+                        bi[h][j] = p.bias ? __ldg(p.bias + n) : 0.0f;
+                    }
+                if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->tmem_full[acc]), acc_phase, abort_flag, to)) {
+                    if (to && lane == 0) report_timeout(p, ctl, tile, 2, 100 + acc);
+                    ok = false;
+                    break;
+                }
+                ptx::tc_fence_after();
+                for (int c = parity; c < chunks; c += 2) {
+                    if (m0 + c * kChunkT >= p.M) break;                     // chunk entirely past the last token
+                    const uint32_t stage = stage0 + buf * kEpiStageBytes;
+                    if (lane == 0) ptx::tma_store_wait_read<1>();           // the store that last read this buffer is done
+                    __syncwarp();
+                    uint32_t v[2][16];
+                    ptx::tmem_ld_16x256b_x4(tbase + (uint32_t)(c * kChunkT), v[0]);
+                    ptx::tmem_ld_16x256b_x4(tbase + (16u << 16) + (uint32_t)(c * kChunkT), v[1]);
+                    ptx::tmem_ld_wait();
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        uint32_t pk[8];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+#pragma unroll
+                            for (int j = 0; j < 2; ++j) {
+                                float y0 = __fmaf_rn(__int2float_rn((int32_t)v[h][4 * i + 2 * j]), sc[h][j], bi[h][j]);
+                                float y1 = __fmaf_rn(__int2float_rn((int32_t)v[h][4 * i + 2 * j + 1]), sc[h][j], bi[h][j]);
+                                if (p.act == GPUSQ_ACT_GELU) {
+                                    y0 = gelu_erfc(y0);
+                                    y1 = gelu_erfc(y1);
+                                }
+                                const __half2 hh = __floats2half2_rn(y0, y1);   // low = token 2(t%4), high = +1
+                                pk[2 * i + j] = *reinterpret_cast<const uint32_t *>(&hh);
+                            }
+                        // matrices of one stmatrix: (tokens 0-7, feat 0-7), (0-7, 8-15), (8-15, 0-7), (8-15, 8-15)
+                        const int mid = lane >> 3, r = lane & 7;
+#pragma unroll
+                        for (int s2 = 0; s2 < 2; ++s2) {
+                            const int tok = 16 * s2 + 8 * (mid >> 1) + r;
+                            const int chunk16 = 2 * h + (mid & 1);
+                            const uint32_t addr = stage + (uint32_t)(tok * 64 + ((chunk16 ^ ((tok >> 1) & 3)) << 4));
+                            ptx::stmatrix_x4_trans(addr, pk[4 * s2 + 0], pk[4 * s2 + 1], pk[4 * s2 + 2], pk[4 * s2 + 3]);
+                        }
+                    }
+                    ptx::fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        ptx::tma_store_2d(&map_y, stage, tn * kBlockF + quarter * 32, (int32_t)(m0 + c * kChunkT));
+                        ptx::tma_store_commit();
+                    }
+                    buf ^= 1u;
+                }
+            } else {
+                const int n = tn * kBlockF + quarter * 32 + lane;      // this thread's output feature
+                float sc = 1.0f, bi = 0.0f;
+                if (p.out_type != GPUSQ_OUT_I32) {
+                    sc = __fmul_rn(__ldg(p.w_scale + n), x_scale);
+                    bi = p.bias ? __ldg(p.bias + n) : 0.0f;
+                }
+                if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->tmem_full[acc]), acc_phase, abort_flag, to)) {
+                    if (to && lane == 0) report_timeout(p, ctl, tile, 2, 100 + acc);
+                    ok = false;
+                    break;
+                }
+                ptx::tc_fence_after();
+                for (int c = parity; c < block_t / 16; c += 2) {
+                    uint32_t r[16];
+                    ptx::tmem_ld_32x32b_x16(tbase + (uint32_t)(c * 16), r);
+                    ptx::tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const int64_t m = m0 + c * 16 + j;
+                        if (m < p.M) {
+                            const int32_t a = (int32_t)r[j];
+                            if (p.out_type == GPUSQ_OUT_I32) {
+                                reinterpret_cast<int32_t *>(p.Y)[m * p.N + n] = a;
                             } else {
+                                float y = __fmaf_rn(__int2float_rn(a), sc, bi);
+                                if (p.act == GPUSQ_ACT_GELU) y = gelu_erfc(y);
                                 int q = __float2int_rn(__fdiv_rn(y, out_scale));
                                 q = max(-127, min(127, q));
                                 reinterpret_cast<int8_t *>(p.Y)[m * p.N + n] = (int8_t)q;
@@ -298,6 +372,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctl->tmem_empty[acc]));
         }
+        // staging buffers must stay valid until the bulk stores have read them
+        if (lane == 0) ptx::tma_store_wait_all<0>();
     }
 
     ptx::tc_fence_before();
@@ -343,16 +419,30 @@ static bool make_map_u8(CUtensorMap *map, const void *base, uint64_t rows, uint6
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Y [M, N] f16 row-major; box = 32 features x 32 tokens, 64-byte swizzle (the staging-tile layout)
+static bool make_map_y_f16(CUtensorMap *map, void *base, uint64_t M, uint64_t N)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {N, M};
+    cuuint64_t strides[1] = {N * 2};
+    cuuint32_t box[2] = {32, (cuuint32_t)kChunkT};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
+           CUDA_SUCCESS;
+}
+
 static int g_block_t_override = 0;
 
-// Tokens per tile: a multiple of 16 up to 240 chosen so that the last wave of
+// Tokens per tile: a multiple of 32 up to 224 chosen so that the last wave of
 // tiles over the SMs is as full as possible (per-tile cost ~ block_t + fixed part).
 static int choose_block_t(int64_t M, int tiles_n, int sms)
 {
     if (g_block_t_override) return g_block_t_override;
-    int best = 240;
+    int best = kMaxBlockT;
     double best_cost = 1e300;
-    for (int bt = 240; bt >= 32; bt -= 16) {
+    for (int bt = kMaxBlockT; bt >= 32; bt -= 32) {
         const int64_t tiles = (int64_t)tiles_n * ceil_div(M, bt);
         const int64_t waves = ceil_div(tiles, sms);
         const double cost = (double)waves * (bt + 48);
@@ -390,6 +480,8 @@ static int launch_gemm(const int8_t *Xq, const void *Wsrc, const float *w_scale,
     else
         ok = make_map_u8(&map_a, Wsrc, (uint64_t)N, (uint64_t)K, 128, kBlockF, CU_TENSOR_MAP_SWIZZLE_128B);
     ok = ok && make_map_u8(&map_b, Xq, (uint64_t)M, (uint64_t)K, 128, (uint32_t)block_t, CU_TENSOR_MAP_SWIZZLE_128B);
+    CUtensorMap map_y = map_b;      // placeholder unless the output is FP16
+    if (out_type == GPUSQ_OUT_F16) ok = ok && make_map_y_f16(&map_y, Y, (uint64_t)M, (uint64_t)N);
     if (!ok) return GPUSQ_ERR_CUDA;
 
     GemmParams p;
@@ -420,7 +512,7 @@ static int launch_gemm(const int8_t *Xq, const void *Wsrc, const float *w_scale,
 
     const int64_t tiles = (int64_t)tiles_n * ceil_div(M, block_t);
     const int grid = (int)(tiles < sms ? tiles : sms);
-    gemm_i8_kernel<kSparse><<<grid, kNumThreads, C::kSmemBytes, (cudaStream_t)stream>>>(map_a, map_b, p);
+    gemm_i8_kernel<kSparse><<<grid, kNumThreads, C::kSmemBytes, (cudaStream_t)stream>>>(map_a, map_b, map_y, p);
     return launch_status();
 }
 
@@ -449,7 +541,7 @@ int gpusq_gemm_i8_dense(const int8_t *Xq, const int8_t *Wq, const float *w_scale
 
 int gpusq_set_block_tokens(int block_t)
 {
-    if (block_t != 0 && (block_t < 16 || block_t > kMaxBlockT || block_t % 16)) return GPUSQ_ERR_ARG;
+    if (block_t != 0 && (block_t < 32 || block_t > kMaxBlockT || block_t % 32)) return GPUSQ_ERR_ARG;
     g_block_t_override = block_t;
     return GPUSQ_OK;
 }

@@ -123,7 +123,7 @@ GEMM_SHAPES = [
 
 
 @pytest.mark.parametrize("M,N,K", GEMM_SHAPES)
-@pytest.mark.parametrize("block_t", [0, 16, 112, 240])
+@pytest.mark.parametrize("block_t", [0, 32, 96, 224])
 def test_spgemm_int32_bit_exact(B, M, N, K, block_t):
     d, prep, Xq, xs = _prep(M + N + K, M, N, K)
     acc_o = oracle.spgemm_acc(Xq, prep["vals"], prep["meta"])
