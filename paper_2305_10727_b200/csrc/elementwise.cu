@@ -266,13 +266,34 @@ act_absmax_kernel(const uint4 *__restrict__ X, uint32_t *__restrict__ partial, i
     if (threadIdx.x == 0) partial[blockIdx.x] = (uint32_t)r;
 }
 
-__device__ __forceinline__ uint32_t quant4_f16(uint32_t lo, uint32_t hi, float s)
+// Same code as quant_code(x, s) without the division: r = x * (1/s) is within 2^-22 |r| of the
+// exactly rounded quotient, so unless r lies within 1e-4 of a rounding boundary (k + 0.5) both
+// round to the same integer; the rare boundary case repeats the step with the true division.
+// (|r| >= 256 saturates to +-127 either way.)
+__device__ __forceinline__ int quant_code_mul(float x, float s, float inv_s)
+{
+    float r = x * inv_s;
+    const float d = fabsf(r - rintf(r));
+    if (d > 0.5f - 1e-4f && fabsf(r) < 256.0f) r = __fdiv_rn(x, s);
+    return __float2int_rn(r);
+}
+
+__device__ __forceinline__ uint32_t pack4_s8_clamp127(int a, int b, int c, int d)
+{
+    // cvt.pack.sat.s8.s32.b32 r, x, y, z  gives  r = (z << 16) | (sat8(x) << 8) | sat8(y)
+    uint32_t hi, out;
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(d), "r"(c), "r"(0));
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(out) : "r"(b), "r"(a), "r"(hi));
+    return __vmaxs4(out, 0x81818181u);     // -128 -> -127
+}
+
+__device__ __forceinline__ uint32_t quant4_f16(uint32_t lo, uint32_t hi, float s, float inv_s)
 {
     const __half2 a = *reinterpret_cast<const __half2 *>(&lo);
     const __half2 b = *reinterpret_cast<const __half2 *>(&hi);
     const float2 fa = __half22float2(a), fb = __half22float2(b);
-    return (uint32_t)(quant_code(fa.x, s) & 0xFF) | ((uint32_t)(quant_code(fa.y, s) & 0xFF) << 8) |
-           ((uint32_t)(quant_code(fb.x, s) & 0xFF) << 16) | ((uint32_t)(quant_code(fb.y, s) & 0xFF) << 24);
+    return pack4_s8_clamp127(quant_code_mul(fa.x, s, inv_s), quant_code_mul(fa.y, s, inv_s),
+                             quant_code_mul(fb.x, s, inv_s), quant_code_mul(fb.y, s, inv_s));
 }
 
 // n_partials > 0: the scale is derived from the partial maxima and written to
@@ -293,16 +314,17 @@ act_quant_kernel(const uint4 *__restrict__ X, uint2 *__restrict__ Xq, float *x_s
     } else {
         s = *x_scale;
     }
+    const float inv_s = __frcp_rn(s);
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     for (; i + stride < vec8; i += 2 * stride) {
         const uint4 v0 = __ldg(X + i), v1 = __ldg(X + i + stride);
-        __stcs(Xq + i, make_uint2(quant4_f16(v0.x, v0.y, s), quant4_f16(v0.z, v0.w, s)));
-        __stcs(Xq + i + stride, make_uint2(quant4_f16(v1.x, v1.y, s), quant4_f16(v1.z, v1.w, s)));
+        Xq[i] = make_uint2(quant4_f16(v0.x, v0.y, s, inv_s), quant4_f16(v0.z, v0.w, s, inv_s));
+        Xq[i + stride] = make_uint2(quant4_f16(v1.x, v1.y, s, inv_s), quant4_f16(v1.z, v1.w, s, inv_s));
     }
     for (; i < vec8; i += stride) {
         const uint4 v = __ldg(X + i);
-        __stcs(Xq + i, make_uint2(quant4_f16(v.x, v.y, s), quant4_f16(v.z, v.w, s)));
+        Xq[i] = make_uint2(quant4_f16(v.x, v.y, s, inv_s), quant4_f16(v.z, v.w, s, inv_s));
     }
 }
 
