@@ -42,7 +42,8 @@ typedef enum gpusq_status {
     GPUSQ_ERR_UNSUPPORTED_ARCH = 5, /* current device is not compute capability 10.x */
     GPUSQ_ERR_CUDA = 6,             /* a CUDA runtime / driver call failed */
     GPUSQ_ERR_TIMEOUT = 7,          /* a bounded device-side wait expired (see status_buf) */
-    GPUSQ_ERR_ARG = 8               /* an enum argument is out of range */
+    GPUSQ_ERR_ARG = 8,              /* an enum argument is out of range */
+    GPUSQ_ERR_TOO_LARGE = 9         /* the tensor exceeds the fixed capacity of a *_static entry point */
 } gpusq_status;
 
 enum { GPUSQ_ACT_NONE = 0, GPUSQ_ACT_GELU = 1 };
@@ -127,6 +128,33 @@ int gpusq_pack24(const int8_t *vals, const uint8_t *meta, void *Wpacked, int N, 
 size_t gpusq_quant_act_workspace(int64_t M, int K);
 int gpusq_quant_act(const void *X, int8_t *Xq, float *x_scale, int scale_mode, int64_t M, int K,
                     void *workspace, size_t ws_bytes, void *stream);
+
+/* ---------------------------------------------------------------------------
+ * gpusq_quant_act_static -- gpusq_quant_act for callers that cannot hand over
+ * scratch memory.  (An addition of this library; the paper has no counterpart.)
+ *
+ * Some hosts of this code may not allocate device memory at the point where
+ * they quantise activations: an inference-server plugin whose enqueue hook
+ * runs after the server has planned and frozen all device memory, a real-time
+ * loop that forbids allocator calls for their unbounded latency, or a process
+ * that was handed a fixed memory budget it does not own.  gpusq_quant_act
+ * needs a small workspace from the caller; this variant needs none.  It uses a
+ * fixed 8 KB array that lives inside the library image on every GPU that loads
+ * the library (held until the process exits) and performs no cudaMalloc,
+ * cudaFree or other allocating call.
+ *
+ * Same arguments and results as gpusq_quant_act, minus workspace / ws_bytes.
+ *   - Capacity: M * K <= 2^32 elements; larger tensors are rejected with
+ *     GPUSQ_ERR_TOO_LARGE and nothing is enqueued.
+ *   - The first call on each device (with that device current) looks up the
+ *     array's device address; make that first call outside any stream capture.
+ *   - All calls on one GPU share the one array: two calls whose kernels can
+ *     overlap on the GPU (different streams, no ordering between them) race
+ *     and may both produce a wrong scale.  Calls ordered on one stream are
+ *     safe; what an earlier call left in the array is never read.
+ */
+int gpusq_quant_act_static(const void *X, int8_t *Xq, float *x_scale, int scale_mode, int64_t M,
+                           int K, void *stream);
 
 /* ---------------------------------------------------------------------------
  * gpusq_spgemm_i8 -- the fused layer: 2:4-sparse INT8 GEMM + epilogue.

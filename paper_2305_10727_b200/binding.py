@@ -24,7 +24,7 @@ SCALE_COMPUTE, SCALE_GIVEN = 0, 1
 EXPORTS = (
     "gpusq_status_string", "gpusq_prune24", "gpusq_quant_weight", "gpusq_compress24",
     "gpusq_decompress24", "gpusq_packed_bytes", "gpusq_pack24", "gpusq_quant_act_workspace",
-    "gpusq_quant_act", "gpusq_spgemm_i8", "gpusq_gemm_i8_dense", "gpusq_set_block_tokens",
+    "gpusq_quant_act", "gpusq_quant_act_static", "gpusq_spgemm_i8", "gpusq_gemm_i8_dense", "gpusq_set_block_tokens",
 )
 
 _lib = None
@@ -59,6 +59,7 @@ def load() -> ctypes.CDLL:
     lib.gpusq_quant_act_workspace.argtypes = [i64, i32]
     lib.gpusq_quant_act_workspace.restype = sz
     lib.gpusq_quant_act.argtypes = [vp, vp, vp, i32, i64, i32, vp, sz, vp]
+    lib.gpusq_quant_act_static.argtypes = [vp, vp, vp, i32, i64, i32, vp]
     gemm_args = [vp, vp, vp, vp, vp, i32, i32, vp, vp, i64, i32, i32, vp, vp]
     lib.gpusq_spgemm_i8.argtypes = gemm_args
     lib.gpusq_gemm_i8_dense.argtypes = gemm_args
@@ -170,6 +171,22 @@ def quant_act(X: torch.Tensor, Xq: Optional[torch.Tensor] = None, x_scale: Optio
     ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     _check(load().gpusq_quant_act(_ptr(X), _ptr(Xq), _ptr(x_scale), scale_mode, M, K, _ptr(workspace),
                                   ws_bytes, _stream()), "gpusq_quant_act")
+    return Xq, x_scale
+
+
+def quant_act_static(X: torch.Tensor, Xq: Optional[torch.Tensor] = None, x_scale: Optional[torch.Tensor] = None,
+                     scale_mode: int = SCALE_COMPUTE):
+    """gpusq_quant_act_static: no workspace argument; the library's own fixed scratch is used."""
+    _dev(X, torch.float16, "X")
+    M, K = X.shape
+    if Xq is None:
+        Xq = torch.empty((M, K), dtype=torch.int8, device=X.device)
+    if x_scale is None:
+        if scale_mode == SCALE_GIVEN:
+            raise ValueError("scale_mode GIVEN needs x_scale")
+        x_scale = torch.empty((1,), dtype=torch.float32, device=X.device)
+    _check(load().gpusq_quant_act_static(_ptr(X), _ptr(Xq), _ptr(x_scale), scale_mode, M, K, _stream()),
+           "gpusq_quant_act_static")
     return Xq, x_scale
 
 

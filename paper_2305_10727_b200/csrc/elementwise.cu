@@ -4,6 +4,8 @@
 // per tensor; no shared-memory staging is needed (no reuse across threads).
 #include <cuda_fp16.h>
 
+#include <mutex>
+
 #include "common.cuh"
 
 namespace gpusq {
@@ -328,6 +330,30 @@ act_quant_kernel(const uint4 *__restrict__ X, uint2 *__restrict__ Xq, float *x_s
     }
 }
 
+// ---- library-owned scratch for gpusq_quant_act_static ----
+// One fixed array per GPU that loads the library (8 KB, held until the process exits).  In host code
+// the symbol below is only a handle: the address the kernels need comes from cudaGetSymbolAddress,
+// looked up once per device with that device current.
+constexpr int64_t kStaticMaxElems = (int64_t)1 << 32;     // largest M*K the static entry point accepts
+static __device__ __align__(256) uint32_t g_act_scratch[kMaxPartials];
+constexpr int kMaxDevices = 64;
+static std::mutex g_scratch_mutex;
+static uint32_t *g_scratch_addr[kMaxDevices] = {};
+
+static int static_scratch(uint32_t **out)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return GPUSQ_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_scratch_mutex);
+    if (!g_scratch_addr[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_act_scratch) != cudaSuccess || !p) return GPUSQ_ERR_CUDA;
+        g_scratch_addr[dev] = static_cast<uint32_t *>(p);
+    }
+    *out = g_scratch_addr[dev];
+    return GPUSQ_OK;
+}
+
 inline int grid_for(int64_t items, int per_sm)
 {
     int64_t blocks = ceil_div(items, kThreads);
@@ -450,6 +476,32 @@ int gpusq_quant_act(const void *X, int8_t *Xq, float *x_scale, int scale_mode, i
     return launch_status();
 }
 
+int gpusq_quant_act_static(const void *X, int8_t *Xq, float *x_scale, int scale_mode, int64_t M, int K,
+                           void *stream)
+{
+    if (!X || !Xq || !x_scale) return GPUSQ_ERR_NULL;
+    if (M <= 0 || K <= 0 || K % 8) return GPUSQ_ERR_SHAPE;
+    if (scale_mode != GPUSQ_SCALE_COMPUTE && scale_mode != GPUSQ_SCALE_GIVEN) return GPUSQ_ERR_ARG;
+    if (M > kStaticMaxElems / K) return GPUSQ_ERR_TOO_LARGE;
+    if (!aligned(X, 16) || !aligned(Xq, 16)) return GPUSQ_ERR_ALIGN;
+    if (int st = check_arch()) return st;
+    uint32_t *scratch = nullptr;
+    if (int st = static_scratch(&scratch)) return st;     // first call on a device resolves the address
+    const int64_t vec8 = M * (int64_t)K / 8;
+    cudaStream_t s = (cudaStream_t)stream;
+    int n_partials = 0;
+    if (scale_mode == GPUSQ_SCALE_COMPUTE) {
+        // every slot that is read below is written here first, so stale contents do not matter
+        n_partials = grid_for(ceil_div(vec8, 4), 8);
+        if (n_partials > kMaxPartials) n_partials = kMaxPartials;
+        act_absmax_kernel<<<n_partials, kThreads, 0, s>>>(reinterpret_cast<const uint4 *>(X), scratch, vec8);
+        if (int st = launch_status()) return st;
+    }
+    act_quant_kernel<<<grid_for(ceil_div(vec8, 2), 8), kThreads, 0, s>>>(
+        reinterpret_cast<const uint4 *>(X), reinterpret_cast<uint2 *>(Xq), x_scale, scratch, n_partials, vec8);
+    return launch_status();
+}
+
 const char *gpusq_status_string(int status)
 {
     switch (status) {
@@ -462,6 +514,7 @@ const char *gpusq_status_string(int status)
     case GPUSQ_ERR_CUDA: return "GPUSQ_ERR_CUDA: a CUDA call failed";
     case GPUSQ_ERR_TIMEOUT: return "GPUSQ_ERR_TIMEOUT: a bounded device-side wait expired";
     case GPUSQ_ERR_ARG: return "GPUSQ_ERR_ARG: an enum argument is out of range";
+    case GPUSQ_ERR_TOO_LARGE: return "GPUSQ_ERR_TOO_LARGE: the tensor exceeds the fixed capacity of this entry point";
     default: return "unknown gpusq status";
     }
 }

@@ -30,7 +30,7 @@ def test_every_declared_symbol_is_exported(lib):
 
 def test_status_strings(lib):
     assert B.status_string(0) == "GPUSQ_OK"
-    for code in range(1, 9):
+    for code in range(1, 10):
         assert B.status_string(code).startswith("GPUSQ_ERR_")
     assert "unknown" in B.status_string(99)
 
@@ -65,6 +65,12 @@ def test_argument_errors_are_reported_before_any_cuda_call(lib):
     assert lib.gpusq_quant_act(p(a16), p(a16), p(a16), 0, 4, 8, p(a16), 8, None) == WS
     assert lib.gpusq_quant_act(p(a16), p(a16), p(a16), 2, 4, 8, p(a16), 1 << 20, None) == ARG
     assert lib.gpusq_quant_act(p(a16), p(a16), p(a16), 1, 4, 12, None, 0, None) == SHAPE
+    TOO_LARGE = 9
+    assert lib.gpusq_quant_act_static(p(a16), p(a16), None, 0, 4, 8, None) == NULL
+    assert lib.gpusq_quant_act_static(p(a16), p(a16), p(a16), 0, 4, 12, None) == SHAPE
+    assert lib.gpusq_quant_act_static(p(a16), p(a16), p(a16), 5, 4, 8, None) == ARG
+    assert lib.gpusq_quant_act_static(p(a16), p(a16), p(a16), 0, (1 << 29) + 1, 8, None) == TOO_LARGE
+    assert lib.gpusq_quant_act_static(p(a16 + 8), p(a16), p(a16), 0, 4, 8, None) == ALIGN
     for fn in (lib.gpusq_spgemm_i8, lib.gpusq_gemm_i8_dense):
         ok = [p(a16), p(a16), p(a16), p(a16), None, 0, 0, None, p(a16), 8, 128, 64, None, None]
         bad = list(ok); bad[0] = None
