@@ -105,7 +105,7 @@ int gpusq_decompress24(const int8_t *vals, const uint8_t *meta, int8_t *Wq, int 
  * Wpacked holds gpusq_packed_bytes(N, K) bytes, 256-byte aligned:
  *   [0, Np*Kp/2)            values, row-major [Np, Kp/2], zero padded
  *   [Np*Kp/2, Np*Kp*5/8)    metadata tiles [Np/128][Kp/128][128 rows][16 bytes]
- * with Np = N rounded up to 128 and Kp = K rounded up to 128.
+ * with Np = N rounded up to 256 and Kp = K rounded up to 128.
  * Requires N > 0, K > 0, K % 8 == 0.
  */
 size_t gpusq_packed_bytes(int N, int K);

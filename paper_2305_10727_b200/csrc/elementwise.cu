@@ -189,6 +189,7 @@ decompress24_kernel(const uint32_t *__restrict__ vals, const uint8_t *__restrict
 }
 
 // -------------------------------------------------------------------- pack
+// Np = N rounded up to 256 (a CTA pair's features), Kp = K rounded up to 128.
 // Values: [Np, Kp/2] zero padded.  Metadata: [Np/128][Kp/128][128 rows][16 bytes],
 // i.e. for each 128-row x 128-column block of W the 16 metadata bytes of a row
 // are contiguous and rows follow each other: the 2 KB block is what one
@@ -424,7 +425,7 @@ int gpusq_decompress24(const int8_t *vals, const uint8_t *meta, int8_t *Wq, int 
 size_t gpusq_packed_bytes(int N, int K)
 {
     if (N <= 0 || K <= 0) return 0;
-    const size_t Np = (size_t)round_up(N, 128), Kp = (size_t)round_up(K, 128);
+    const size_t Np = (size_t)round_up(N, 256), Kp = (size_t)round_up(K, 128);
     return Np * Kp / 2 + Np * Kp / 8;
 }
 
@@ -434,7 +435,7 @@ int gpusq_pack24(const int8_t *vals, const uint8_t *meta, void *Wpacked, int N, 
     if (N <= 0 || K <= 0 || K % 8) return GPUSQ_ERR_SHAPE;
     if (!aligned(vals, 4) || !aligned(Wpacked, 256)) return GPUSQ_ERR_ALIGN;
     if (int st = check_arch()) return st;
-    const int Np = round_up(N, 128), Kp = round_up(K, 128);
+    const int Np = round_up(N, 256), Kp = round_up(K, 128);
     const int64_t chunks = (int64_t)Np * (Kp / 32) + (int64_t)Np * (Kp / 128);
     pack24_kernel<<<grid_for(chunks, 8), kThreads, 0, (cudaStream_t)stream>>>(
         vals, meta, reinterpret_cast<uint8_t *>(Wpacked), N, K, Np, Kp);

@@ -3,24 +3,37 @@
 // tensor memory, and the de-quantise / bias / GELU / convert epilogue.
 //
 // Orientation.  The layer is Y[M,N] = X[M,K] * W[N,K]^T.  tcgen05.mma.sp wants
-// the sparse operand as MMA-A, so the kernel computes Y^T = W * X^T:
-//   MMA-M = 128 output features (one tensor-memory lane each),
-//   MMA-N = block_t tokens (one 32-bit tensor-memory column each),
-//   MMA-K = 64 (sparse) or 32 (dense) per instruction, 128 per pipeline stage.
+// the sparse operand as MMA-A, so the kernel computes Y^T = W * X^T.
 //
-// One persistent CTA per SM, ten warps:
-//   warp 0    TMA producer (one elected lane): W values, W metadata, X tile
-//   warp 1    tensor-memory owner and MMA issuer (one elected lane)
-//   warps 2-9 epilogue: two warps per 32-lane quarter of tensor memory, which
-//             take alternate 32-token chunks of the tile
+// CTA pairs.  Two CTAs on neighbouring SMs (a cluster of two) work on one
+// output tile of 256 features x block_t tokens with cta_group::2 instructions:
+//   MMA-M = 256: each CTA supplies its own 128 features of W (values and, for
+//           the sparse variant, metadata) and keeps their accumulators in its
+//           own tensor memory (one lane per feature);
+//   MMA-N = block_t tokens (one 32-bit tensor-memory column each): each CTA
+//           loads only half of the tile's activation rows, the instruction
+//           reads both halves;
+//   MMA-K = 64 (sparse) or 32 (dense) per instruction, 128 per pipeline stage.
+// Sharing the activation tile halves the L2 -> shared-memory traffic per
+// output and keeps the sparse instruction's operand reads within the
+// shared-memory bandwidth of one SM.
+//
+// Persistent clusters (one per SM pair), ten warps per CTA:
+//   warp 0    TMA producer (one elected lane), in both CTAs; every load of a
+//             stage counts its bytes on the full barrier of the pair's CTA 0
+//   warp 1    tensor-memory owner (both CTAs); in CTA 0 one elected lane
+//             issues the MMAs for the pair and signals barriers in both CTAs
+//   warps 2-9 epilogue: each warp owns 16 tensor-memory lanes (features);
+//             four warps (64 features) share a staging tile and a TMA store
 // Stages are handed over with mbarriers (full/empty per smem stage,
 // full/empty per accumulator buffer); two accumulator buffers let the
 // epilogue of tile i overlap the main loop of tile i+1.
 //
-// FP16 epilogue: tcgen05.ld in the 16x256b (accumulator-fragment) shape, FP32
-// math, pack pairs of tokens to f16x2, stmatrix.trans into a 64-byte-swizzled
-// [32 tokens][32 features] staging tile per warp, TMA store to Y (full 64-byte
-// row segments, rows beyond M clipped by the tensor map).
+// FP16 epilogue: tcgen05.ld in the 16x256b (accumulator-fragment) shape with
+// the next chunk's load in flight during the arithmetic, FP32 math, pairs of
+// tokens packed to f16x2, stmatrix.trans into a 128-byte-swizzled
+// [32 tokens][64 features] staging tile, TMA store to Y (full 128-byte row
+// segments; rows beyond M and features beyond N clipped by the tensor map).
 #include <cuda.h>
 #include <cuda_fp16.h>
 
@@ -31,31 +44,37 @@
 
 namespace gpusq {
 
-constexpr int kBlockF = 128;        // features per tile
+constexpr int kBlockF = 128;        // features per CTA and tile
+constexpr int kPairF = 2 * kBlockF; // features per CTA pair and tile
 constexpr int kBlockK = 128;        // K per stage
 constexpr int kMaxBlockT = 224;     // tokens per tile (runtime value, multiple of 32)
 constexpr int kChunkT = 32;         // tokens per epilogue chunk
 constexpr int kEpiWarps = 8;
 constexpr int kNumThreads = 64 + 32 * kEpiWarps;
 constexpr int kTmemCols = 512;
-constexpr int kAccStride = 224;     // column offset of the second accumulator
-constexpr int kMetaCol = 448;       // metadata slots: 4 columns per stage from here
-constexpr int kEpiStageBytes = kChunkT * 64;          // [32 tokens][32 features] f16
-constexpr int kEpiBytes = kEpiWarps * 2 * kEpiStageBytes;
+constexpr int kAccStride = 256;     // column offset of the second accumulator
+constexpr int kMetaCol = 224;       // metadata slots: 4 columns per stage from here (below the second accumulator)
+constexpr int kEpiGroups = 2;       // groups of four epilogue warps, 64 features each
+constexpr int kEpiBufs = 4;         // staging tiles per group
+constexpr int kEpiBufBytes = kChunkT * 128;           // [32 tokens][64 features] f16
+constexpr int kEpiBytes = kEpiGroups * kEpiBufs * kEpiBufBytes;
 
 template <bool kSparse>
 struct Cfg {
     static constexpr int kABytes = kSparse ? kBlockF * 64 : kBlockF * 128;
-    static constexpr int kBBytes = kMaxBlockT * 128;
+    static constexpr int kBBytes = (kMaxBlockT / 2) * 128;       // this CTA's half of the token rows
     static constexpr int kMetaBytes = kSparse ? 2048 : 0;
     static constexpr int kStageBytes = kABytes + kBBytes + kMetaBytes;
-    static constexpr int kStages = kSparse ? 5 : 4;
+    static constexpr int kStages = kSparse ? 8 : 6;
     static constexpr int kCtlBytes = 1024;
     static constexpr int kSmemBytes = kStages * kStageBytes + kEpiBytes + kCtlBytes + 1024 /* alignment slack */;
     static constexpr int kMmasPerStage = kSparse ? 2 : 4;
     static constexpr int kAStepBytes = 32;                    // per MMA along K, both variants
     static constexpr int kBStepBytes = kSparse ? 64 : 32;
     static constexpr int kASwizzle = kSparse ? 64 : 128;
+    static_assert(kStageBytes % 1024 == 0, "stages keep the 1024-byte alignment of the swizzled tiles");
+    static_assert(kStages <= 8, "eight metadata slots below the second accumulator");
+    static_assert(kSmemBytes <= 232448, "shared memory per CTA");
 };
 
 struct Ctl {
@@ -69,7 +88,6 @@ struct Ctl {
 };
 
 struct GemmParams {
-    const uint8_t *meta;        // packed metadata tiles (sparse only)
     const float *w_scale;
     const float *x_scale;
     const float *bias;
@@ -84,9 +102,13 @@ struct GemmParams {
     int out_type;
 };
 
+// A wait of this CTA expired: raise the abort flag in both CTAs of the pair and record where.
 __device__ __forceinline__ void report_timeout(const GemmParams &p, Ctl *ctl, int tile, int role, int stage)
 {
-    if (atomicExch(&ctl->abort_flag, 1u) == 0u && p.status) {
+    const uint32_t flag = ptx::smem_u32(&ctl->abort_flag);
+    const bool first = atomicExch(&ctl->abort_flag, 1u) == 0u;
+    ptx::st_cluster_u32(ptx::map_to_cta(flag, ptx::cluster_ctarank() ^ 1u), 1u);
+    if (first && p.status) {
         if (atomicCAS(p.status, 0, GPUSQ_ERR_TIMEOUT) == 0) {
             p.status[1] = tile;
             p.status[2] = role;
@@ -136,13 +158,14 @@ __device__ __forceinline__ float gelu_one(float y)
 }
 
 template <bool kSparse>
-__global__ void __launch_bounds__(kNumThreads, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kNumThreads, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-               const __grid_constant__ CUtensorMap map_y, const GemmParams p)
+               const __grid_constant__ CUtensorMap map_e, const __grid_constant__ CUtensorMap map_y,
+               const GemmParams p)
 {
     using C = Cfg<kSparse>;
     extern __shared__ uint8_t smem_raw[];
-    // operand tiles need 1024-byte alignment for the 128-byte swizzle
+    // operand tiles need 1024-byte alignment for the 128-byte swizzle; both CTAs of a pair get the same offsets
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t *epi_smem = smem + C::kStages * C::kStageBytes;
     Ctl *ctl = reinterpret_cast<Ctl *>(epi_smem + kEpiBytes);
@@ -150,12 +173,17 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
+    const uint32_t rank = ptx::cluster_ctarank();            // 0 issues the MMAs of the pair
+    const int cluster_id = blockIdx.x >> 1;
+    const int num_clusters = gridDim.x >> 1;
     const int block_t = p.block_t;
-    const int tiles_n = p.N / kBlockF;
+    const int half_t = block_t >> 1;
+    const int tiles_n = (p.N + kPairF - 1) / kPairF;
     const int tiles_m = (int)((p.M + block_t - 1) / block_t);
     const int num_tiles = tiles_n * tiles_m;
     const int num_kb = (p.K + kBlockK - 1) / kBlockK;
-    const uint32_t stage_tx = (uint32_t)(C::kABytes + block_t * 128 + C::kMetaBytes);
+    // bytes both CTAs together bring in per stage
+    const uint32_t stage_tx = 2u * (uint32_t)(C::kABytes + half_t * 128 + C::kMetaBytes);
 
     auto a_smem = [&](int s) { return smem + s * C::kStageBytes; };
     auto b_smem = [&](int s) { return smem + s * C::kStageBytes + C::kABytes; };
@@ -168,21 +196,23 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
         for (int a = 0; a < 2; ++a) {
             ptx::mbar_init(ptx::smem_u32(&ctl->tmem_full[a]), 1);
-            ptx::mbar_init(ptx::smem_u32(&ctl->tmem_empty[a]), kEpiWarps);
+            ptx::mbar_init(ptx::smem_u32(&ctl->tmem_empty[a]), 2 * kEpiWarps);   // the epilogue warps of both CTAs
         }
         ptx::mbar_init(ptx::smem_u32(&ctl->drain), 1);
         ctl->abort_flag = 0;
         ptx::fence_barrier_init();
         ptx::prefetch_tensormap(&map_a);
         ptx::prefetch_tensormap(&map_b);
+        if (kSparse) ptx::prefetch_tensormap(&map_e);
         if (p.out_type == GPUSQ_OUT_F16) ptx::prefetch_tensormap(&map_y);
     }
     if (warp == 1) {
-        ptx::tmem_alloc(ptx::smem_u32(&ctl->tmem_base), kTmemCols);
-        ptx::tmem_relinquish();
+        ptx::tmem_alloc_pair(ptx::smem_u32(&ctl->tmem_base), kTmemCols);
+        ptx::tmem_relinquish_pair();
     }
     ptx::tc_fence_before();
     __syncthreads();
+    ptx::cluster_sync();            // the other CTA's barriers exist before anything is signalled on them
     ptx::tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
 
@@ -194,8 +224,10 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             uint32_t issued = 0;            // bit s: a load into stage s was issued
             uint32_t last_parity = 0;       // bit s: parity of the last phase issued into stage s
             bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+            for (int tile = cluster_id; ok && tile < num_tiles; tile += num_clusters) {
                 const int tn = tile % tiles_n, tm = tile / tiles_n;
+                const int f0 = tn * kPairF + (int)rank * kBlockF;             // this CTA's first feature
+                const int t0 = tm * block_t + (int)rank * half_t;             // this CTA's first token row
                 for (int kb = 0; kb < num_kb; ++kb) {
                     bool to;
                     if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag, to)) {
@@ -203,14 +235,15 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         ok = false;
                         break;
                     }
-                    const uint32_t bar = ptx::smem_u32(&ctl->full[stage]);
-                    ptx::mbar_arrive_expect_tx(bar, stage_tx);
-                    ptx::tma_load_2d(ptx::smem_u32(a_smem(stage)), &map_a, bar,
-                                     kb * (kSparse ? 64 : 128), tn * kBlockF);
-                    ptx::tma_load_2d(ptx::smem_u32(b_smem(stage)), &map_b, bar, kb * kBlockK, tm * block_t);
+                    // all bytes of the stage, from both CTAs, are counted on CTA 0's barrier
+                    const uint32_t bar = ptx::map_to_cta(ptx::smem_u32(&ctl->full[stage]), 0);
+                    if (rank == 0) ptx::mbar_arrive_expect_tx(ptx::smem_u32(&ctl->full[stage]), stage_tx);
+                    ptx::tma_load_2d_pair(ptx::smem_u32(a_smem(stage)), &map_a, bar, kb * (kSparse ? 64 : 128), f0);
+                    ptx::tma_load_2d_pair(ptx::smem_u32(b_smem(stage)), &map_b, bar, kb * kBlockK, t0);
                     if (kSparse) {
-                        const uint8_t *src = p.meta + ((int64_t)tn * num_kb + kb) * 2048;
-                        ptx::bulk_load(ptx::smem_u32(m_smem(stage)), src, 2048, bar);
+                        // 2 KB metadata block of (feature tile, k block) = 8 rows of 256 bytes
+                        ptx::tma_load_2d_pair(ptx::smem_u32(m_smem(stage)), &map_e, bar, 0,
+                                              ((f0 / kBlockF) * num_kb + kb) * 8);
                     }
                     issued |= 1u << stage;
                     last_parity = (last_parity & ~(1u << stage)) | (phase << stage);
@@ -220,8 +253,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     }
                 }
             }
-            if (*abort_flag) {
-                // do not leave while bulk copies may still land in this CTA's shared memory
+            if (*abort_flag && rank == 0) {
+                // do not leave while bulk copies may still land in the pair's shared memory
                 for (int s = 0; s < C::kStages; ++s) {
                     if (issued & (1u << s)) {
                         uint32_t none = 0;
@@ -233,13 +266,13 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
     } else if (warp == 1) {
         // ---------------------------------------------------------- MMA issuer
-        if (ptx::elect_one()) {
-            const uint32_t idesc = ptx::make_idesc_i8(kBlockF, block_t, kSparse);
+        if (rank == 0 && ptx::elect_one()) {
+            const uint32_t idesc = ptx::make_idesc_i8(kPairF, block_t, kSparse);
             int stage = 0;
             uint32_t phase = 0;
             int local = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++local) {
+            for (int tile = cluster_id; ok && tile < num_tiles; tile += num_clusters, ++local) {
                 const int acc = local & 1;
                 const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
                 bool to;
@@ -259,7 +292,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     ptx::tc_fence_after();
                     const uint32_t meta_t = tmem_base + (uint32_t)(kMetaCol + 4 * stage);
                     if (kSparse) {
-                        ptx::tc_cp_128x128b(meta_t, ptx::make_smem_desc(ptx::smem_u32(m_smem(stage)), 128, 0));
+                        ptx::tc_cp_128x128b_pair(meta_t, ptx::make_smem_desc(ptx::smem_u32(m_smem(stage)), 128, 0));
                     }
                     const uint64_t adesc = ptx::make_smem_desc(ptx::smem_u32(a_smem(stage)), C::kASwizzle * 8, C::kASwizzle);
                     const uint64_t bdesc = ptx::make_smem_desc(ptx::smem_u32(b_smem(stage)), 1024, 128);
@@ -269,17 +302,18 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         const uint64_t bd = bdesc + (uint64_t)((k * C::kBStepBytes) >> 4);
                         const uint32_t accum = (kb | k) != 0 ? 1u : 0u;
                         if (kSparse)
-                            ptx::tc_mma_sp_i8(d_tmem, ad, bd, meta_t + 2u * k, idesc, accum);
+                            ptx::tc_mma_sp_i8_pair(d_tmem, ad, bd, meta_t + 2u * k, idesc, accum);
                         else
-                            ptx::tc_mma_i8(d_tmem, ad, bd, idesc, accum);
+                            ptx::tc_mma_i8_pair(d_tmem, ad, bd, idesc, accum);
                     }
-                    ptx::tc_commit(ptx::smem_u32(&ctl->empty[stage]));   // stage reusable once these MMAs are done
+                    // the stage is reusable in both CTAs once these MMAs are done
+                    ptx::tc_commit_pair(ptx::smem_u32(&ctl->empty[stage]), 3);
                     if (++stage == C::kStages) {
                         stage = 0;
                         phase ^= 1u;
                     }
                 }
-                if (ok) ptx::tc_commit(ptx::smem_u32(&ctl->tmem_full[acc]));
+                if (ok) ptx::tc_commit_pair(ptx::smem_u32(&ctl->tmem_full[acc]), 3);
             }
             if (*abort_flag) {
                 // let every MMA issued so far retire before tensor memory is released
@@ -291,97 +325,125 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
     } else {
         // ------------------------------------------------------------ epilogue
-        const int quarter = warp & 3;                      // tensor-memory lanes [32q, 32q+32)
-        const int parity = (warp - 2) >> 2;                // this warp takes chunks parity, parity+2, ...
+        const int quarter = warp & 3;                      // tensor-memory lanes [32q, 32q+32) are this warp's to read
+        const int half = (warp - 2) >> 2;                  // which 16 of them (F16 path) / which chunks (other paths)
         const float x_scale = (p.out_type == GPUSQ_OUT_I32) ? 1.0f : __ldg(p.x_scale);
         const float out_scale = (p.out_type == GPUSQ_OUT_I8) ? __ldg(p.out_scale) : 1.0f;
-        const uint32_t stage0 = ptx::smem_u32(epi_smem + (warp - 2) * 2 * kEpiStageBytes);
+        // the accumulators of both CTAs are released on CTA 0's barrier, where the MMA issuer waits
+        const uint32_t tmem_empty0 = ptx::map_to_cta(ptx::smem_u32(&ctl->tmem_empty[0]), 0);
+        const uint32_t tmem_empty1 = ptx::map_to_cta(ptx::smem_u32(&ctl->tmem_empty[1]), 0);
+        const int group = quarter >> 1;                    // features [64 group, 64 group + 64) of the CTA's 128
+        const uint32_t group_bar = 1u + (uint32_t)group;
+        const bool store_leader = half == 0 && (quarter & 1) == 0 && lane == 0;
+        const uint32_t stage0 = ptx::smem_u32(epi_smem + group * kEpiBufs * kEpiBufBytes);
         const int chunks = block_t / kChunkT;
         uint32_t buf = 0;
         int local = 0;
-        bool ok = true;
-        for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++local) {
+        for (int tile = cluster_id; tile < num_tiles; tile += num_clusters, ++local) {
             const int tn = tile % tiles_n, tm = tile / tiles_n;
             const int acc = local & 1;
             const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
             const int64_t m0 = (int64_t)tm * block_t;
-            const uint32_t tbase = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * kAccStride);
+            const int n0 = tn * kPairF + (int)rank * kBlockF;
+            const bool n_valid = n0 < p.N;                 // the pair's second CTA may lie past the last feature
+            const uint32_t tmem_empty = acc ? tmem_empty1 : tmem_empty0;
             bool to;
             if (p.out_type == GPUSQ_OUT_F16) {
-                // features of this thread: 32q + 16h + 8j + lane/4 (h = lane half of the quarter, j = fragment row)
-                float sc[2][2], bi[2][2];
+                // features of this thread: n0 + 32q + 16 half + 8j + lane/4 (j = fragment row)
+                float sc[2], bi[2];
 #pragma unroll
-                for (int h = 0; h < 2; ++h)
-#pragma unroll
-                    for (int j = 0; j < 2; ++j) {
-                        const int n = tn * kBlockF + quarter * 32 + 16 * h + 8 * j + (lane >> 2);
-                        sc[h][j] = __fmul_rn(__ldg(p.w_scale + n), x_scale);
-                        bi[h][j] = p.bias ? __ldg(p.bias + n) : 0.0f;
-                    }
-                if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->tmem_full[acc]), acc_phase, abort_flag, to)) {
-                    if (to && lane == 0) report_timeout(p, ctl, tile, 2, 100 + acc);
-                    ok = false;
-                    break;
+                for (int j = 0; j < 2; ++j) {
+                    const int n = n0 + quarter * 32 + 16 * half + 8 * j + (lane >> 2);
+                    sc[j] = n_valid ? __fmul_rn(__ldg(p.w_scale + n), x_scale) : 0.0f;
+                    bi[j] = (n_valid && p.bias) ? __ldg(p.bias + n) : 0.0f;
                 }
+                const bool got = ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->tmem_full[acc]), acc_phase, abort_flag, to);
+                if (!got && to && lane == 0) report_timeout(p, ctl, tile, 2, 100 + acc);
+                // the four warps of a group leave together or not at all (they share named barriers below)
+                if (!ptx::bar_and(group_bar, 128, got)) break;
                 ptx::tc_fence_after();
-                for (int c = parity; c < chunks; c += 2) {
-                    if (m0 + c * kChunkT >= p.M) break;                     // chunk entirely past the last token
-                    const uint32_t stage = stage0 + buf * kEpiStageBytes;
-                    if (lane == 0) ptx::tma_store_wait_read<1>();           // the store that last read this buffer is done
+                int nchunks = 0;
+                if (n_valid) {
+                    const int64_t left = p.M - m0;         // > 0
+                    nchunks = left >= block_t ? chunks : (int)((left + kChunkT - 1) / kChunkT);
+                }
+                const uint32_t tbase =
+                    tmem_base + ((uint32_t)(quarter * 32 + half * 16) << 16) + (uint32_t)(acc * kAccStride);
+                const int chunk16 = 4 * (quarter & 1) + 2 * half;      // 16-byte column of this warp's first feature
+
+                auto release = [&]() {
+                    ptx::tc_fence_before();
                     __syncwarp();
-                    uint32_t v[2][16];
-                    ptx::tmem_ld_16x256b_x4(tbase + (uint32_t)(c * kChunkT), v[0]);
-                    ptx::tmem_ld_16x256b_x4(tbase + (16u << 16) + (uint32_t)(c * kChunkT), v[1]);
-                    ptx::tmem_ld_wait();
+                    if (lane == 0) ptx::mbar_arrive_cluster(tmem_empty);
+                };
+                // one chunk: v holds it (load issued earlier), vn receives the next one
+                auto step = [&](uint32_t(&v)[16], uint32_t(&vn)[16], int c) {
+                    ptx::tmem_ld_wait_regs(v);
+                    if (c + 1 < nchunks)
+                        ptx::tmem_ld_16x256b_x4(tbase + (uint32_t)((c + 1) * kChunkT), vn);
+                    else
+                        release();                                     // every column of this tile is in registers
+                    uint32_t pk[8];
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        uint32_t pk[8];
+                    for (int i = 0; i < 4; ++i)
 #pragma unroll
-                        for (int i = 0; i < 4; ++i)
-#pragma unroll
-                            for (int j = 0; j < 2; ++j) {
-                                float2 y = __ffma2_rn(make_float2(__int2float_rn((int32_t)v[h][4 * i + 2 * j]),
-                                                                  __int2float_rn((int32_t)v[h][4 * i + 2 * j + 1])),
-                                                      make_float2(sc[h][j], sc[h][j]), make_float2(bi[h][j], bi[h][j]));
-                                if (p.act == GPUSQ_ACT_GELU) y = gelu_pair(y);
-                                const __half2 hh = __floats2half2_rn(y.x, y.y);   // low = token 2(t%4), high = +1
-                                pk[2 * i + j] = *reinterpret_cast<const uint32_t *>(&hh);
-                            }
-                        // matrices of one stmatrix: (tokens 0-7, feat 0-7), (0-7, 8-15), (8-15, 0-7), (8-15, 8-15)
-                        const int mid = lane >> 3, r = lane & 7;
-#pragma unroll
-                        for (int s2 = 0; s2 < 2; ++s2) {
-                            const int tok = 16 * s2 + 8 * (mid >> 1) + r;
-                            const int chunk16 = 2 * h + (mid & 1);
-                            const uint32_t addr = stage + (uint32_t)(tok * 64 + ((chunk16 ^ ((tok >> 1) & 3)) << 4));
-                            ptx::stmatrix_x4_trans(addr, pk[4 * s2 + 0], pk[4 * s2 + 1], pk[4 * s2 + 2], pk[4 * s2 + 3]);
+                        for (int j = 0; j < 2; ++j) {
+                            float2 y = __ffma2_rn(make_float2(__int2float_rn((int32_t)v[4 * i + 2 * j]),
+                                                              __int2float_rn((int32_t)v[4 * i + 2 * j + 1])),
+                                                  make_float2(sc[j], sc[j]), make_float2(bi[j], bi[j]));
+                            if (p.act == GPUSQ_ACT_GELU) y = gelu_pair(y);
+                            const __half2 hh = __floats2half2_rn(y.x, y.y);   // low = token 2(t%4), high = +1
+                            pk[2 * i + j] = *reinterpret_cast<const uint32_t *>(&hh);
                         }
+                    // matrices of one stmatrix: (tokens 0-7, feat 0-7), (0-7, 8-15), (8-15, 0-7), (8-15, 8-15)
+                    const uint32_t stage = stage0 + buf * kEpiBufBytes;
+                    const int mid = lane >> 3, r = lane & 7;
+#pragma unroll
+                    for (int s2 = 0; s2 < 2; ++s2) {
+                        const int tok = 16 * s2 + 8 * (mid >> 1) + r;
+                        const int c16 = chunk16 + (mid & 1);
+                        const uint32_t addr = stage + (uint32_t)(tok * 128 + ((c16 ^ (tok & 7)) << 4));
+                        ptx::stmatrix_x4_trans(addr, pk[4 * s2 + 0], pk[4 * s2 + 1], pk[4 * s2 + 2], pk[4 * s2 + 3]);
                     }
                     ptx::fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0) {
-                        ptx::tma_store_2d(&map_y, stage, tn * kBlockF + quarter * 32, (int32_t)(m0 + c * kChunkT));
+                    // staging tile `buf + 1` is written after the next barrier: its last store must have read it
+                    if (store_leader) ptx::tma_store_wait_read<kEpiBufs - 2>();
+                    ptx::bar_sync(group_bar, 128);
+                    if (store_leader) {
+                        ptx::tma_store_2d(&map_y, stage, n0 + group * 64, (int32_t)(m0 + c * kChunkT));
                         ptx::tma_store_commit();
                     }
-                    buf ^= 1u;
+                    buf = (buf + 1 == (uint32_t)kEpiBufs) ? 0u : buf + 1;
+                };
+
+                if (nchunks == 0) {
+                    release();
+                } else {
+                    uint32_t v0[16], v1[16];
+                    ptx::tmem_ld_16x256b_x4(tbase, v0);
+                    for (int c = 0; c < nchunks; c += 2) {
+                        step(v0, v1, c);
+                        if (c + 1 < nchunks) step(v1, v0, c + 1);
+                    }
                 }
             } else {
-                const int n = tn * kBlockF + quarter * 32 + lane;      // this thread's output feature
+                const int n = n0 + quarter * 32 + lane;                // this thread's output feature
                 float sc = 1.0f, bi = 0.0f;
-                if (p.out_type != GPUSQ_OUT_I32) {
+                if (p.out_type != GPUSQ_OUT_I32 && n_valid) {
                     sc = __fmul_rn(__ldg(p.w_scale + n), x_scale);
                     bi = p.bias ? __ldg(p.bias + n) : 0.0f;
                 }
                 if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->tmem_full[acc]), acc_phase, abort_flag, to)) {
                     if (to && lane == 0) report_timeout(p, ctl, tile, 2, 100 + acc);
-                    ok = false;
                     break;
                 }
                 ptx::tc_fence_after();
-                for (int c = parity; c < block_t / 16; c += 2) {
+                const uint32_t tbase = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * kAccStride);
+                for (int c = half; c < block_t / 16 && n_valid; c += 2) {
+                    if (m0 + c * 16 >= p.M) break;
                     uint32_t r[16];
                     ptx::tmem_ld_32x32b_x16(tbase + (uint32_t)(c * 16), r);
-                    ptx::tmem_ld_wait();
+                    ptx::tmem_ld_wait_regs(r);
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
                         const int64_t m = m0 + c * 16 + j;
@@ -399,20 +461,22 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         }
                     }
                 }
+                ptx::tc_fence_before();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive_cluster(tmem_empty);
             }
-            ptx::tc_fence_before();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctl->tmem_empty[acc]));
         }
-        // staging buffers must stay valid until the bulk stores have read them
-        if (lane == 0) ptx::tma_store_wait_all<0>();
+        // staging tiles must stay valid until the bulk stores have read them
+        if (store_leader) ptx::tma_store_wait_all<0>();
     }
 
+    // neither CTA leaves while the other may still signal its barriers or read its shared memory
     ptx::tc_fence_before();
     __syncthreads();
+    ptx::cluster_sync();
     if (warp == 1) {
         ptx::tc_fence_after();
-        ptx::tmem_dealloc(tmem_base, kTmemCols);
+        ptx::tmem_dealloc_pair(tmem_base, kTmemCols);
     }
 }
 
@@ -451,32 +515,32 @@ static bool make_map_u8(CUtensorMap *map, const void *base, uint64_t rows, uint6
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Y [M, N] f16 row-major; box = 32 features x 32 tokens, 64-byte swizzle (the staging-tile layout)
+// Y [M, N] f16 row-major; box = 64 features x 32 tokens, 128-byte swizzle (the staging-tile layout)
 static bool make_map_y_f16(CUtensorMap *map, void *base, uint64_t M, uint64_t N)
 {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     cuuint64_t dims[2] = {N, M};
     cuuint64_t strides[1] = {N * 2};
-    cuuint32_t box[2] = {32, (cuuint32_t)kChunkT};
+    cuuint32_t box[2] = {64, (cuuint32_t)kChunkT};
     cuuint32_t estr[2] = {1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-              CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
            CUDA_SUCCESS;
 }
 
 static int g_block_t_override = 0;
 
 // Tokens per tile: a multiple of 32 up to 224 chosen so that the last wave of
-// tiles over the SMs is as full as possible (per-tile cost ~ block_t + fixed part).
-static int choose_block_t(int64_t M, int tiles_n, int sms)
+// tiles over the SM pairs is as full as possible (per-tile cost ~ block_t + fixed part).
+static int choose_block_t(int64_t M, int tiles_n, int clusters)
 {
     if (g_block_t_override) return g_block_t_override;
     int best = kMaxBlockT;
     double best_cost = 1e300;
     for (int bt = kMaxBlockT; bt >= 32; bt -= 32) {
         const int64_t tiles = (int64_t)tiles_n * ceil_div(M, bt);
-        const int64_t waves = ceil_div(tiles, sms);
+        const int64_t waves = ceil_div(tiles, clusters);
         const double cost = (double)waves * (bt + 48);
         if (cost < best_cost * 0.999) {
             best_cost = cost;
@@ -484,6 +548,30 @@ static int choose_block_t(int64_t M, int tiles_n, int sms)
         }
     }
     return best;
+}
+
+// SM pairs that can hold one cluster of this kernel each, per device (0 = unknown yet)
+template <bool kSparse>
+static int max_clusters(int sms)
+{
+    static std::mutex mu;
+    static int cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return sms / 2;
+    std::lock_guard<std::mutex> lock(mu);
+    if (cached[dev] == 0) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(sms & ~1), 1, 1);
+        cfg.blockDim = dim3(kNumThreads, 1, 1);
+        cfg.dynamicSmemBytes = Cfg<kSparse>::kSmemBytes;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, gemm_i8_kernel<kSparse>, &cfg) != cudaSuccess || n <= 0) {
+            (void)cudaGetLastError();
+            n = sms / 2;
+        }
+        cached[dev] = n < sms / 2 ? n : sms / 2;
+    }
+    return cached[dev];
 }
 
 template <bool kSparse>
@@ -500,10 +588,23 @@ static int launch_gemm(const int8_t *Xq, const void *Wsrc, const float *w_scale,
     if (!aligned(Xq, 16) || !aligned(Wsrc, 16) || !aligned(Y, 16)) return GPUSQ_ERR_ALIGN;
     if (int st = check_arch()) return st;
 
+    static std::once_flag attr_once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(attr_once, [] {
+        attr_err = cudaFuncSetAttribute(gemm_i8_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        Cfg<true>::kSmemBytes);
+        if (attr_err == cudaSuccess)
+            attr_err = cudaFuncSetAttribute(gemm_i8_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            Cfg<false>::kSmemBytes);
+    });
+    if (attr_err != cudaSuccess) return GPUSQ_ERR_CUDA;
+
     const int sms = num_sms();
-    const int tiles_n = N / kBlockF;
-    const int block_t = choose_block_t(M, tiles_n, sms);
-    const int Kp = round_up(K, 128), Np = round_up(N, 128);
+    const int clusters = max_clusters<kSparse>(sms);
+    if (clusters <= 0) return GPUSQ_ERR_CUDA;
+    const int tiles_n = (N + kPairF - 1) / kPairF;
+    const int block_t = choose_block_t(M, tiles_n, clusters);
+    const int Kp = round_up(K, 128), Np = round_up(N, kPairF);
 
     CUtensorMap map_a, map_b;
     bool ok;
@@ -511,13 +612,20 @@ static int launch_gemm(const int8_t *Xq, const void *Wsrc, const float *w_scale,
         ok = make_map_u8(&map_a, Wsrc, (uint64_t)Np, (uint64_t)Kp / 2, 64, kBlockF, CU_TENSOR_MAP_SWIZZLE_64B);
     else
         ok = make_map_u8(&map_a, Wsrc, (uint64_t)N, (uint64_t)K, 128, kBlockF, CU_TENSOR_MAP_SWIZZLE_128B);
-    ok = ok && make_map_u8(&map_b, Xq, (uint64_t)M, (uint64_t)K, 128, (uint32_t)block_t, CU_TENSOR_MAP_SWIZZLE_128B);
+    ok = ok && make_map_u8(&map_b, Xq, (uint64_t)M, (uint64_t)K, 128, (uint32_t)(block_t / 2),
+                           CU_TENSOR_MAP_SWIZZLE_128B);
+    CUtensorMap map_e = map_b;      // placeholder unless the weight is sparse
+    if (kSparse) {
+        // metadata blocks of 2 KB, viewed as 8 rows of 256 bytes each
+        const uint8_t *meta = reinterpret_cast<const uint8_t *>(Wsrc) + (size_t)Np * (Kp / 2);
+        ok = ok && make_map_u8(&map_e, meta, (uint64_t)(Np / 128) * (Kp / 128) * 8, 256, 256, 8,
+                               CU_TENSOR_MAP_SWIZZLE_NONE);
+    }
     CUtensorMap map_y = map_b;      // placeholder unless the output is FP16
     if (out_type == GPUSQ_OUT_F16) ok = ok && make_map_y_f16(&map_y, Y, (uint64_t)M, (uint64_t)N);
     if (!ok) return GPUSQ_ERR_CUDA;
 
     GemmParams p;
-    p.meta = kSparse ? reinterpret_cast<const uint8_t *>(Wsrc) + (size_t)Np * (Kp / 2) : nullptr;
     p.w_scale = w_scale;
     p.x_scale = x_scale;
     p.bias = bias;
@@ -531,20 +639,9 @@ static int launch_gemm(const int8_t *Xq, const void *Wsrc, const float *w_scale,
     p.act = act;
     p.out_type = out_type;
 
-    static std::once_flag attr_once;
-    static cudaError_t attr_err = cudaSuccess;
-    std::call_once(attr_once, [] {
-        attr_err = cudaFuncSetAttribute(gemm_i8_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        Cfg<true>::kSmemBytes);
-        if (attr_err == cudaSuccess)
-            attr_err = cudaFuncSetAttribute(gemm_i8_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            Cfg<false>::kSmemBytes);
-    });
-    if (attr_err != cudaSuccess) return GPUSQ_ERR_CUDA;
-
     const int64_t tiles = (int64_t)tiles_n * ceil_div(M, block_t);
-    const int grid = (int)(tiles < sms ? tiles : sms);
-    gemm_i8_kernel<kSparse><<<grid, kNumThreads, C::kSmemBytes, (cudaStream_t)stream>>>(map_a, map_b, map_y, p);
+    const int grid = 2 * (int)(tiles < clusters ? tiles : clusters);
+    gemm_i8_kernel<kSparse><<<grid, kNumThreads, C::kSmemBytes, (cudaStream_t)stream>>>(map_a, map_b, map_e, map_y, p);
     return launch_status();
 }
 

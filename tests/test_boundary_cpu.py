@@ -39,7 +39,7 @@ def test_size_queries(lib):
     # values K/2 bytes + metadata K/8 bytes per row, both padded to 128 x 128 blocks
     assert B.packed_bytes(768, 768) == 768 * 768 * 5 // 8
     assert B.packed_bytes(768, 192) == 768 * 256 * 5 // 8
-    assert B.packed_bytes(100, 64) == 128 * 128 * 5 // 8
+    assert B.packed_bytes(100, 64) == 256 * 128 * 5 // 8
     assert B.packed_bytes(0, 64) == 0
     assert B.quant_act_workspace(12608, 768) >= 16
 

@@ -74,7 +74,7 @@ def test_compress_decompress_pack(B, N, K):
     assert np.array_equal(B.decompress24(vals, meta).cpu().numpy(), Wq)
     # packed blob: zero-padded values, then metadata blocks [N/128][K/128][128][16]
     blob = B.pack24(vals, meta).cpu().numpy()
-    Np, Kp = -(-N // 128) * 128, -(-K // 128) * 128
+    Np, Kp = -(-N // 256) * 256, -(-K // 128) * 128     # rows padded to a CTA pair's 256 features
     assert blob.size == B.packed_bytes(N, K) == Np * Kp * 5 // 8
     pv = blob[:Np * Kp // 2].view(np.int8).reshape(Np, Kp // 2)
     assert np.array_equal(pv[:N, :K // 2], vals_o) and not pv[N:].any() and not pv[:, K // 2:].any()
