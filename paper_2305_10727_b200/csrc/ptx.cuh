@@ -56,22 +56,26 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t byt
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
                  : "memory");
 }
+// One try: the hardware parks the thread until the phase completes or about `kSuspendNs` have passed,
+// so a waiting warp issues an instruction every microsecond or so instead of competing for issue
+// slots with the warps that have work (a dozen polling warps otherwise take half of an SM's slots).
+constexpr uint32_t kSuspendNs = 1000;
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 {
     uint32_t ok;
     asm volatile(
         "{\n"
         ".reg .pred P;\n"
-        "mbarrier.try_wait.parity.shared::cta.b64 P, [%1], %2;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 P, [%1], %2, %3;\n"
         "selp.u32 %0, 1, 0, P;\n"
         "}\n"
         : "=r"(ok)
-        : "r"(bar), "r"(parity)
+        : "r"(bar), "r"(parity), "r"(kSuspendNs)
         : "memory");
     return ok != 0;
 }
 
-// Bounded wait: gives up after `limit_ns` of wall time, or as soon as another
+// Bounded wait: gives up after `kWaitLimitNs` of wall time, or as soon as another
 // thread of the CTA has raised *abort_flag.  Returns false on either; the
 // caller that timed out raises the flag itself.
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s
@@ -79,18 +83,14 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
                                                   volatile uint32_t *abort_flag, bool &timed_out)
 {
     timed_out = false;
-    uint64_t t0 = 0;
-    for (uint32_t it = 0;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = globaltimer_ns();
+    for (;;) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 63u) == 63u) {
-            if (*abort_flag) return false;
-            const uint64_t now = globaltimer_ns();
-            if (t0 == 0) {
-                t0 = now;
-            } else if (now - t0 > kWaitLimitNs) {
-                timed_out = true;
-                return false;
-            }
+        if (*abort_flag) return false;
+        if (globaltimer_ns() - t0 > kWaitLimitNs) {
+            timed_out = true;
+            return false;
         }
     }
 }
@@ -243,7 +243,9 @@ __device__ __forceinline__ void cluster_sync()
 // arrive on an mbarrier of any CTA of the cluster (address from map_to_cta)
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
 {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+    // default semantics (release at CTA scope): a cluster-scope release would first drain this thread's
+    // global and shared stores, which costs over a thousand cycles while the memory system is loaded
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 __device__ __forceinline__ void st_cluster_u32(uint32_t cluster_addr, uint32_t v)
 {
