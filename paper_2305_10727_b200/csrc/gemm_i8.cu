@@ -18,15 +18,21 @@
 // output and keeps the sparse instruction's operand reads within the
 // shared-memory bandwidth of one SM.
 //
-// Persistent clusters (one per SM pair), ten warps per CTA:
-//   warp 0    TMA producer (one elected lane), in both CTAs; every load of a
-//             stage counts its bytes on the full barrier of the pair's CTA 0
-//   warp 1    tensor-memory owner (both CTAs); in CTA 0 one elected lane
-//             issues the MMAs for the pair and signals barriers in both CTAs
-//   warps 2-9 epilogue: each warp owns 16 tensor-memory lanes (features);
-//             four warps (64 features) share a staging tile and a TMA store
-// Stages are handed over with mbarriers (full/empty per smem stage,
-// full/empty per accumulator buffer); two accumulator buffers let the
+// Persistent clusters (one per SM pair), twenty warps per CTA:
+//   warp 0      TMA producer (one elected lane), in both CTAs; every load of a
+//               stage counts its bytes on the full barrier of the pair's CTA 0
+//   warp 1      tensor-memory owner (both CTAs); in CTA 0 one elected lane
+//               issues the MMAs for the pair and signals barriers in both CTAs
+//   warps 2-17  epilogue: each warp owns 16 tensor-memory lanes (features) and
+//               every other 32-token chunk; four warps (64 features) fill one
+//               staging tile per chunk.  The work on a chunk is short and
+//               latency-bound, so several warps per scheduler are needed to
+//               keep the issue slots busy
+//   warps 18-19 one elected lane each issues the TMA stores of one 64-feature
+//               half's staging tiles and recycles them
+// Everything is handed over with mbarriers (full/empty per smem stage,
+// full/empty per accumulator buffer, full/free per staging tile), so no warp
+// waits for another one's instruction stream; two accumulator buffers let the
 // epilogue of tile i overlap the main loop of tile i+1.
 //
 // FP16 epilogue: tcgen05.ld in the 16x256b (accumulator-fragment) shape with
@@ -49,13 +55,14 @@ constexpr int kPairF = 2 * kBlockF; // features per CTA pair and tile
 constexpr int kBlockK = 128;        // K per stage
 constexpr int kMaxBlockT = 224;     // tokens per tile (runtime value, multiple of 32)
 constexpr int kChunkT = 32;         // tokens per epilogue chunk
-constexpr int kEpiWarps = 8;
-constexpr int kNumThreads = 64 + 32 * kEpiWarps;
+constexpr int kEpiWarps = 16;
+constexpr int kStoreWarp0 = 2 + kEpiWarps;   // first of the two store warps
+constexpr int kNumThreads = 32 * (kStoreWarp0 + 2);
 constexpr int kTmemCols = 512;
 constexpr int kAccStride = 256;     // column offset of the second accumulator
 constexpr int kMetaCol = 224;       // metadata slots: 4 columns per stage from here (below the second accumulator)
-constexpr int kEpiGroups = 2;       // groups of four epilogue warps, 64 features each
-constexpr int kEpiBufs = 4;         // staging tiles per group
+constexpr int kEpiGroups = 4;       // groups of four epilogue warps: 64 features x every other chunk
+constexpr int kEpiBufs = 3;         // staging tiles per group
 constexpr int kEpiBufBytes = kChunkT * 128;           // [32 tokens][64 features] f16
 constexpr int kEpiBytes = kEpiGroups * kEpiBufs * kEpiBufBytes;
 
@@ -65,7 +72,7 @@ struct Cfg {
     static constexpr int kBBytes = (kMaxBlockT / 2) * 128;       // this CTA's half of the token rows
     static constexpr int kMetaBytes = kSparse ? 2048 : 0;
     static constexpr int kStageBytes = kABytes + kBBytes + kMetaBytes;
-    static constexpr int kStages = kSparse ? 8 : 6;
+    static constexpr int kStages = kSparse ? 7 : 5;
     static constexpr int kCtlBytes = 1024;
     static constexpr int kSmemBytes = kStages * kStageBytes + kEpiBytes + kCtlBytes + 1024 /* alignment slack */;
     static constexpr int kMmasPerStage = kSparse ? 2 : 4;
@@ -83,6 +90,8 @@ struct Ctl {
     uint64_t tmem_full[2];
     uint64_t tmem_empty[2];
     uint64_t drain;
+    uint64_t stg_full[kEpiGroups][kEpiBufs];     // staging tile written by its four warps
+    uint64_t stg_free[kEpiGroups][kEpiBufs];     // staging tile read by its TMA store
     uint32_t tmem_base;
     uint32_t abort_flag;
 };
@@ -199,6 +208,11 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             ptx::mbar_init(ptx::smem_u32(&ctl->tmem_empty[a]), 2 * kEpiWarps);   // the epilogue warps of both CTAs
         }
         ptx::mbar_init(ptx::smem_u32(&ctl->drain), 1);
+        for (int g = 0; g < kEpiGroups; ++g)
+            for (int b = 0; b < kEpiBufs; ++b) {
+                ptx::mbar_init(ptx::smem_u32(&ctl->stg_full[g][b]), 4);
+                ptx::mbar_init(ptx::smem_u32(&ctl->stg_free[g][b]), 1);
+            }
         ctl->abort_flag = 0;
         ptx::fence_barrier_init();
         ptx::prefetch_tensormap(&map_a);
@@ -323,44 +337,104 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 (void)ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->drain), 0, &none, to);
             }
         }
+    } else if (warp >= kStoreWarp0) {
+        // --------------------------------------------------------- TMA stores
+        // One lane per 64-feature half: waits for a staging tile to be filled, stores it, and hands
+        // tiles back to the epilogue warps once the stores have read them.
+        if (p.out_type == GPUSQ_OUT_F16 && ptx::elect_one()) {
+            const int fgroup = warp - kStoreWarp0;         // features [64 fgroup, 64 fgroup + 64) of the CTA's 128
+            const int chunks = block_t / kChunkT;
+            uint32_t filled0 = 0, filled1 = 0;             // staging tiles stored so far, per chunk parity group
+            uint32_t prev1 = 0, prev2 = 0;                 // free barriers of the last two stores (0 = none)
+            int local = 0;
+            bool ok = true;
+            for (int tile = cluster_id; ok && tile < num_tiles; tile += num_clusters, ++local) {
+                const int tn = tile % tiles_n, tm = tile / tiles_n;
+                const int64_t m0 = (int64_t)tm * block_t;
+                const int n0 = tn * kPairF + (int)rank * kBlockF;
+                if (n0 >= p.N) continue;
+                const int64_t left = p.M - m0;
+                const int nchunks = left >= block_t ? chunks : (int)((left + kChunkT - 1) / kChunkT);
+                for (int c = 0; c < nchunks; ++c) {
+                    const int par = (c + local) & 1;       // the group of warps that fills this chunk
+                    const int gi = fgroup * 2 + par;
+                    const uint32_t count = par ? filled1 : filled0;
+                    const uint32_t b = count % kEpiBufs;
+                    bool to;
+                    if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->stg_full[gi][b]), (count / kEpiBufs) & 1u,
+                                                abort_flag, to)) {
+                        if (to) report_timeout(p, ctl, tile, 3, gi * 8 + (int)b);
+                        ok = false;
+                        break;
+                    }
+                    ptx::tma_store_2d(&map_y, ptx::smem_u32(epi_smem + (gi * kEpiBufs + (int)b) * kEpiBufBytes),
+                                      n0 + fgroup * 64, (int32_t)(m0 + c * kChunkT));
+                    ptx::tma_store_commit();
+                    // all but the two newest stores have read their tiles: hand the third newest back
+                    ptx::tma_store_wait_read<2>();
+                    if (prev2) ptx::mbar_arrive(prev2);
+                    prev2 = prev1;
+                    prev1 = ptx::smem_u32(&ctl->stg_free[gi][b]);
+                    if (par) ++filled1; else ++filled0;
+                }
+            }
+            // the staging tiles must stay valid until the bulk stores have read them, and the
+            // stores must be complete before the kernel ends
+            ptx::tma_store_wait_all<0>();
+        }
     } else {
         // ------------------------------------------------------------ epilogue
         const int quarter = warp & 3;                      // tensor-memory lanes [32q, 32q+32) are this warp's to read
-        const int half = (warp - 2) >> 2;                  // which 16 of them (F16 path) / which chunks (other paths)
+        const int half = ((warp - 2) >> 2) & 1;            // which 16 of them (F16 path)
+        const int par = (warp - 2) >> 3;                   // which chunks: every other one
         const float x_scale = (p.out_type == GPUSQ_OUT_I32) ? 1.0f : __ldg(p.x_scale);
         const float out_scale = (p.out_type == GPUSQ_OUT_I8) ? __ldg(p.out_scale) : 1.0f;
         // the accumulators of both CTAs are released on CTA 0's barrier, where the MMA issuer waits
         const uint32_t tmem_empty0 = ptx::map_to_cta(ptx::smem_u32(&ctl->tmem_empty[0]), 0);
         const uint32_t tmem_empty1 = ptx::map_to_cta(ptx::smem_u32(&ctl->tmem_empty[1]), 0);
-        const int group = quarter >> 1;                    // features [64 group, 64 group + 64) of the CTA's 128
-        const uint32_t group_bar = 1u + (uint32_t)group;
-        const bool store_leader = half == 0 && (quarter & 1) == 0 && lane == 0;
+        const int group = (quarter >> 1) * 2 + par;        // 64 features x chunk parity: the warps sharing staging tiles
         const uint32_t stage0 = ptx::smem_u32(epi_smem + group * kEpiBufs * kEpiBufBytes);
         const int chunks = block_t / kChunkT;
-        uint32_t buf = 0;
+        uint32_t filled = 0;                               // staging tiles this warp's group has filled so far
         int local = 0;
-        for (int tile = cluster_id; tile < num_tiles; tile += num_clusters, ++local) {
-            const int tn = tile % tiles_n, tm = tile / tiles_n;
-            const int acc = local & 1;
-            const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
-            const int64_t m0 = (int64_t)tm * block_t;
-            const int n0 = tn * kPairF + (int)rank * kBlockF;
-            const bool n_valid = n0 < p.N;                 // the pair's second CTA may lie past the last feature
-            const uint32_t tmem_empty = acc ? tmem_empty1 : tmem_empty0;
-            bool to;
-            if (p.out_type == GPUSQ_OUT_F16) {
-                // features of this thread: n0 + 32q + 16 half + 8j + lane/4 (j = fragment row)
+        bool ok = true;
+
+        if (p.out_type == GPUSQ_OUT_F16) {
+            // features of this thread: n0 + 32q + 16 half + 8j + lane/4 (j = fragment row)
+            const int nofs = quarter * 32 + 16 * half + (lane >> 2);
+            const int chunk16 = 4 * (quarter & 1) + 2 * half;          // 16-byte column of this warp's first feature
+            // scale and bias of a tile are fetched one tile ahead: the loads are in flight during a whole tile
+            float ws_next[2] = {0.0f, 0.0f}, bi_next[2] = {0.0f, 0.0f};
+            auto fetch = [&](int tile) {
+                const int n0 = (tile % tiles_n) * kPairF + (int)rank * kBlockF;
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                    const bool in = tile < num_tiles && n0 < p.N;
+                    ws_next[j] = in ? __ldg(p.w_scale + n0 + nofs + 8 * j) : 0.0f;
+                    bi_next[j] = (in && p.bias) ? __ldg(p.bias + n0 + nofs + 8 * j) : 0.0f;
+                }
+            };
+            fetch(cluster_id);
+            for (int tile = cluster_id; ok && tile < num_tiles; tile += num_clusters, ++local) {
+                const int tn = tile % tiles_n, tm = tile / tiles_n;
+                const int acc = local & 1;
+                const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
+                const int64_t m0 = (int64_t)tm * block_t;
+                const int n0 = tn * kPairF + (int)rank * kBlockF;
+                const bool n_valid = n0 < p.N;             // the pair's second CTA may lie past the last feature
+                const uint32_t tmem_empty = acc ? tmem_empty1 : tmem_empty0;
                 float sc[2], bi[2];
 #pragma unroll
                 for (int j = 0; j < 2; ++j) {
-                    const int n = n0 + quarter * 32 + 16 * half + 8 * j + (lane >> 2);
-                    sc[j] = n_valid ? __fmul_rn(__ldg(p.w_scale + n), x_scale) : 0.0f;
-                    bi[j] = (n_valid && p.bias) ? __ldg(p.bias + n) : 0.0f;
+                    sc[j] = __fmul_rn(ws_next[j], x_scale);
+                    bi[j] = bi_next[j];
                 }
-                const bool got = ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->tmem_full[acc]), acc_phase, abort_flag, to);
-                if (!got && to && lane == 0) report_timeout(p, ctl, tile, 2, 100 + acc);
-                // the four warps of a group leave together or not at all (they share named barriers below)
-                if (!ptx::bar_and(group_bar, 128, got)) break;
+                fetch(tile + num_clusters);
+                bool to;
+                if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->tmem_full[acc]), acc_phase, abort_flag, to)) {
+                    if (to && lane == 0) report_timeout(p, ctl, tile, 2, 100 + acc);
+                    break;
+                }
                 ptx::tc_fence_after();
                 int nchunks = 0;
                 if (n_valid) {
@@ -369,20 +443,19 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 }
                 const uint32_t tbase =
                     tmem_base + ((uint32_t)(quarter * 32 + half * 16) << 16) + (uint32_t)(acc * kAccStride);
-                const int chunk16 = 4 * (quarter & 1) + 2 * half;      // 16-byte column of this warp's first feature
 
                 auto release = [&]() {
                     ptx::tc_fence_before();
                     __syncwarp();
                     if (lane == 0) ptx::mbar_arrive_cluster(tmem_empty);
                 };
-                // one chunk: v holds it (load issued earlier), vn receives the next one
+                // one chunk: v holds it (load issued earlier), vn receives this warp's next one
                 auto step = [&](uint32_t(&v)[16], uint32_t(&vn)[16], int c) {
                     ptx::tmem_ld_wait_regs(v);
-                    if (c + 1 < nchunks)
-                        ptx::tmem_ld_16x256b_x4(tbase + (uint32_t)((c + 1) * kChunkT), vn);
+                    if (c + 2 < nchunks)
+                        ptx::tmem_ld_16x256b_x4(tbase + (uint32_t)((c + 2) * kChunkT), vn);
                     else
-                        release();                                     // every column of this tile is in registers
+                        release();                                     // all this warp reads of the tile is in registers
                     uint32_t pk[8];
 #pragma unroll
                     for (int i = 0; i < 4; ++i)
@@ -395,8 +468,16 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                             const __half2 hh = __floats2half2_rn(y.x, y.y);   // low = token 2(t%4), high = +1
                             pk[2 * i + j] = *reinterpret_cast<const uint32_t *>(&hh);
                         }
+                    // the staging tile's previous contents have been stored
+                    const uint32_t b = filled % kEpiBufs;
+                    if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->stg_free[group][b]),
+                                                ((filled / kEpiBufs) & 1u) ^ 1u, abort_flag, to)) {
+                        if (to && lane == 0) report_timeout(p, ctl, tile, 2, 200 + (int)b);
+                        ok = false;
+                        return;
+                    }
                     // matrices of one stmatrix: (tokens 0-7, feat 0-7), (0-7, 8-15), (8-15, 0-7), (8-15, 8-15)
-                    const uint32_t stage = stage0 + buf * kEpiBufBytes;
+                    const uint32_t stage = stage0 + b * kEpiBufBytes;
                     const int mid = lane >> 3, r = lane & 7;
 #pragma unroll
                     for (int s2 = 0; s2 < 2; ++s2) {
@@ -405,41 +486,49 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         const uint32_t addr = stage + (uint32_t)(tok * 128 + ((c16 ^ (tok & 7)) << 4));
                         ptx::stmatrix_x4_trans(addr, pk[4 * s2 + 0], pk[4 * s2 + 1], pk[4 * s2 + 2], pk[4 * s2 + 3]);
                     }
-                    ptx::fence_proxy_async_smem();
-                    // staging tile `buf + 1` is written after the next barrier: its last store must have read it
-                    if (store_leader) ptx::tma_store_wait_read<kEpiBufs - 2>();
-                    ptx::bar_sync(group_bar, 128);
-                    if (store_leader) {
-                        ptx::tma_store_2d(&map_y, stage, n0 + group * 64, (int32_t)(m0 + c * kChunkT));
-                        ptx::tma_store_commit();
-                    }
-                    buf = (buf + 1 == (uint32_t)kEpiBufs) ? 0u : buf + 1;
+                    ptx::fence_proxy_async_smem();                     // this lane's writes, for the TMA store
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctl->stg_full[group][b]));
+                    ++filled;
                 };
 
-                if (nchunks == 0) {
+                // this warp's chunks of the tile: c0, c0 + 2, ...; the two parity groups swap every tile
+                const int c0 = (par + local) & 1;
+                if (c0 >= nchunks) {
                     release();
                 } else {
                     uint32_t v0[16], v1[16];
-                    ptx::tmem_ld_16x256b_x4(tbase, v0);
-                    for (int c = 0; c < nchunks; c += 2) {
+                    ptx::tmem_ld_16x256b_x4(tbase + (uint32_t)(c0 * kChunkT), v0);
+                    for (int c = c0; ok && c < nchunks; c += 4) {
                         step(v0, v1, c);
-                        if (c + 1 < nchunks) step(v1, v0, c + 1);
+                        if (ok && c + 2 < nchunks) step(v1, v0, c + 2);
                     }
                 }
-            } else {
+            }
+        } else {
+            for (int tile = cluster_id; tile < num_tiles; tile += num_clusters, ++local) {
+                const int tn = tile % tiles_n, tm = tile / tiles_n;
+                const int acc = local & 1;
+                const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
+                const int64_t m0 = (int64_t)tm * block_t;
+                const int n0 = tn * kPairF + (int)rank * kBlockF;
+                const bool n_valid = n0 < p.N;
+                const uint32_t tmem_empty = acc ? tmem_empty1 : tmem_empty0;
                 const int n = n0 + quarter * 32 + lane;                // this thread's output feature
                 float sc = 1.0f, bi = 0.0f;
                 if (p.out_type != GPUSQ_OUT_I32 && n_valid) {
                     sc = __fmul_rn(__ldg(p.w_scale + n), x_scale);
                     bi = p.bias ? __ldg(p.bias + n) : 0.0f;
                 }
+                bool to;
                 if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->tmem_full[acc]), acc_phase, abort_flag, to)) {
                     if (to && lane == 0) report_timeout(p, ctl, tile, 2, 100 + acc);
                     break;
                 }
                 ptx::tc_fence_after();
                 const uint32_t tbase = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * kAccStride);
-                for (int c = half; c < block_t / 16 && n_valid; c += 2) {
+                // the four warps of a quarter take every fourth 16-token chunk
+                for (int c = (warp - 2) >> 2; c < block_t / 16 && n_valid; c += kEpiWarps / 4) {
                     if (m0 + c * 16 >= p.M) break;
                     uint32_t r[16];
                     ptx::tmem_ld_32x32b_x16(tbase + (uint32_t)(c * 16), r);
@@ -466,8 +555,6 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 if (lane == 0) ptx::mbar_arrive_cluster(tmem_empty);
             }
         }
-        // staging tiles must stay valid until the bulk stores have read them
-        if (store_leader) ptx::tma_store_wait_all<0>();
     }
 
     // neither CTA leaves while the other may still signal its barriers or read its shared memory
