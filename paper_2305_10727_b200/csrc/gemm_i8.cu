@@ -166,6 +166,163 @@ __device__ __forceinline__ float gelu_one(float y)
     return gelu_pair(make_float2(y, y)).x;
 }
 
+// FP16 epilogue of one worker warp.  The warp owns 16 tensor-memory lanes (features) and every
+// other 32-token chunk of each tile.  Per chunk: wait for the chunk's tcgen05.ld (issued one chunk
+// ahead), issue the next one, convert / scale / activate 16 values per thread, wait for a free
+// staging tile, two stmatrix, proxy fence, arrive on the tile's full barrier.  The loop is written
+// for few instructions per chunk: whatever can be precomputed or advanced incrementally is.
+struct EpiF16 {
+    const GemmParams *p;
+    Ctl *ctl;
+    uint32_t tmem_base, stage0, stg_full0, stg_free0, tmem_empty0, tmem_empty1;
+    float x_scale;
+    int warp, lane, rank, cluster_id, num_clusters, tiles_n, num_tiles, block_t;
+
+    // staging-tile ring of this warp's group
+    uint32_t buf_addr, full_bar, free_bar, buf_idx, free_parity;
+    uint32_t stm_off;          // this lane's stmatrix row address inside a staging tile (second one: + 2048)
+    float2 sc2[2], bi2[2];     // scale and bias of this thread's two features, duplicated for packed math
+
+    __device__ __forceinline__ void release(int acc)
+    {
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive_cluster(acc ? tmem_empty1 : tmem_empty0);
+    }
+
+    // One chunk held in v (its load was issued earlier).  next_taddr != 0: issue this warp's next
+    // load into vn; otherwise v was the warp's last chunk of the tile and the accumulator is released.
+    template <bool kGelu>
+    __device__ __forceinline__ bool step(uint32_t (&v)[16], uint32_t (&vn)[16], uint32_t next_taddr, int acc,
+                                         int tile)
+    {
+        ptx::tmem_ld_wait_regs(v);
+        if (next_taddr)
+            ptx::tmem_ld_16x256b_x4(next_taddr, vn);
+        else
+            release(acc);
+        uint32_t pk[8];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                float2 y = __ffma2_rn(make_float2(__int2float_rn((int32_t)v[4 * i + 2 * j]),
+                                                  __int2float_rn((int32_t)v[4 * i + 2 * j + 1])),
+                                      sc2[j], bi2[j]);
+                if (kGelu) y = gelu_pair(y);
+                const __half2 hh = __floats2half2_rn(y.x, y.y);   // low = token 2(t%4), high = +1
+                pk[2 * i + j] = *reinterpret_cast<const uint32_t *>(&hh);
+            }
+        // the staging tile's previous contents have been stored
+        bool to;
+        if (!ptx::mbar_wait_bounded(free_bar, free_parity, &ctl->abort_flag, to)) {
+            if (to && lane == 0) report_timeout(*p, ctl, tile, 2, 200 + (int)buf_idx);
+            return false;
+        }
+        // matrices of one stmatrix: (tokens 0-7, feat 0-7), (0-7, 8-15), (8-15, 0-7), (8-15, 8-15)
+        ptx::stmatrix_x4_trans(buf_addr + stm_off, pk[0], pk[1], pk[2], pk[3]);
+        ptx::stmatrix_x4_trans(buf_addr + stm_off + 2048u, pk[4], pk[5], pk[6], pk[7]);
+        ptx::fence_proxy_async_smem();                     // this lane's writes, for the TMA store
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(full_bar);
+        if (++buf_idx == (uint32_t)kEpiBufs) {
+            buf_idx = 0;
+            free_parity ^= 1u;
+            buf_addr = stage0;
+            full_bar = stg_full0;
+            free_bar = stg_free0;
+        } else {
+            buf_addr += kEpiBufBytes;
+            full_bar += 8;
+            free_bar += 8;
+        }
+        return true;
+    }
+
+    template <bool kGelu>
+    __device__ __forceinline__ void run()
+    {
+        const int quarter = warp & 3;                      // tensor-memory lanes [32q, 32q+32) are this warp's to read
+        const int half = ((warp - 2) >> 2) & 1;            // which 16 of them
+        const int par = (warp - 2) >> 3;                   // which chunks: every other one
+        const int nofs = quarter * 32 + 16 * half + (lane >> 2);       // this thread's first feature in the CTA's 128
+        {
+            // stmatrix row of this lane: token 8 (mid / 2) + r of the tile, 16-byte column c16 (128-byte swizzle)
+            const int mid = lane >> 3, r = lane & 7;
+            const int tok = 8 * (mid >> 1) + r;
+            const int c16 = 4 * (quarter & 1) + 2 * half + (mid & 1);
+            stm_off = (uint32_t)(tok * 128 + ((c16 ^ r) << 4));
+        }
+        buf_addr = stage0;
+        full_bar = stg_full0;
+        free_bar = stg_free0;
+        buf_idx = 0;
+        free_parity = 1;                                   // first round: the tiles are free
+        const int chunks = block_t / kChunkT;
+        const int64_t M = p->M;
+        const int N = p->N;
+        const float *w_scale = p->w_scale, *bias = p->bias;
+
+        // scale and bias of a tile are fetched one tile ahead: the loads are in flight during a whole tile
+        float ws_next[2], bi_next[2];
+        auto fetch = [&](int tile) {
+            const int n0 = (tile % tiles_n) * kPairF + rank * kBlockF;
+            const bool in = tile < num_tiles && n0 < N;
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                ws_next[j] = in ? __ldg(w_scale + n0 + nofs + 8 * j) : 0.0f;
+                bi_next[j] = (in && bias) ? __ldg(bias + n0 + nofs + 8 * j) : 0.0f;
+            }
+        };
+        fetch(cluster_id);
+        int local = 0;
+        for (int tile = cluster_id; tile < num_tiles; tile += num_clusters, ++local) {
+            const int tn = tile % tiles_n, tm = tile / tiles_n;
+            const int acc = local & 1;
+            const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
+            const int64_t m0 = (int64_t)tm * block_t;
+            const bool n_valid = tn * kPairF + rank * kBlockF < N;     // the pair's second CTA may lie past the last feature
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                const float sc = __fmul_rn(ws_next[j], x_scale);
+                sc2[j] = make_float2(sc, sc);
+                bi2[j] = make_float2(bi_next[j], bi_next[j]);
+            }
+            fetch(tile + num_clusters);
+            bool to;
+            if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->tmem_full[acc]), acc_phase, &ctl->abort_flag, to)) {
+                if (to && lane == 0) report_timeout(*p, ctl, tile, 2, 100 + acc);
+                return;
+            }
+            ptx::tc_fence_after();
+            int nchunks = 0;
+            if (n_valid) {
+                const int64_t left = M - m0;               // > 0
+                nchunks = left >= block_t ? chunks : (int)((left + kChunkT - 1) / kChunkT);
+            }
+            // this warp's chunks of the tile: c0, c0 + 2, ...; the two parity groups swap every tile
+            const int c0 = (par + local) & 1;
+            int mine = (nchunks - c0 + 1) >> 1;            // how many of them
+            if (mine <= 0) {
+                release(acc);
+                continue;
+            }
+            uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32 + half * 16) << 16) +
+                             (uint32_t)(acc * kAccStride + c0 * kChunkT);
+            uint32_t v0[16], v1[16];
+            ptx::tmem_ld_16x256b_x4(taddr, v0);
+            for (;;) {
+                taddr += 2 * kChunkT;
+                if (!step<kGelu>(v0, v1, --mine ? taddr : 0u, acc, tile)) return;
+                if (!mine) break;
+                taddr += 2 * kChunkT;
+                if (!step<kGelu>(v1, v0, --mine ? taddr : 0u, acc, tile)) return;
+                if (!mine) break;
+            }
+        }
+    }
+};
+
 template <bool kSparse>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kNumThreads, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
@@ -394,117 +551,31 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const uint32_t tmem_empty1 = ptx::map_to_cta(ptx::smem_u32(&ctl->tmem_empty[1]), 0);
         const int group = (quarter >> 1) * 2 + par;        // 64 features x chunk parity: the warps sharing staging tiles
         const uint32_t stage0 = ptx::smem_u32(epi_smem + group * kEpiBufs * kEpiBufBytes);
-        const int chunks = block_t / kChunkT;
-        uint32_t filled = 0;                               // staging tiles this warp's group has filled so far
         int local = 0;
-        bool ok = true;
 
         if (p.out_type == GPUSQ_OUT_F16) {
-            // features of this thread: n0 + 32q + 16 half + 8j + lane/4 (j = fragment row)
-            const int nofs = quarter * 32 + 16 * half + (lane >> 2);
-            const int chunk16 = 4 * (quarter & 1) + 2 * half;          // 16-byte column of this warp's first feature
-            // scale and bias of a tile are fetched one tile ahead: the loads are in flight during a whole tile
-            float ws_next[2] = {0.0f, 0.0f}, bi_next[2] = {0.0f, 0.0f};
-            auto fetch = [&](int tile) {
-                const int n0 = (tile % tiles_n) * kPairF + (int)rank * kBlockF;
-#pragma unroll
-                for (int j = 0; j < 2; ++j) {
-                    const bool in = tile < num_tiles && n0 < p.N;
-                    ws_next[j] = in ? __ldg(p.w_scale + n0 + nofs + 8 * j) : 0.0f;
-                    bi_next[j] = (in && p.bias) ? __ldg(p.bias + n0 + nofs + 8 * j) : 0.0f;
-                }
-            };
-            fetch(cluster_id);
-            for (int tile = cluster_id; ok && tile < num_tiles; tile += num_clusters, ++local) {
-                const int tn = tile % tiles_n, tm = tile / tiles_n;
-                const int acc = local & 1;
-                const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
-                const int64_t m0 = (int64_t)tm * block_t;
-                const int n0 = tn * kPairF + (int)rank * kBlockF;
-                const bool n_valid = n0 < p.N;             // the pair's second CTA may lie past the last feature
-                const uint32_t tmem_empty = acc ? tmem_empty1 : tmem_empty0;
-                float sc[2], bi[2];
-#pragma unroll
-                for (int j = 0; j < 2; ++j) {
-                    sc[j] = __fmul_rn(ws_next[j], x_scale);
-                    bi[j] = bi_next[j];
-                }
-                fetch(tile + num_clusters);
-                bool to;
-                if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->tmem_full[acc]), acc_phase, abort_flag, to)) {
-                    if (to && lane == 0) report_timeout(p, ctl, tile, 2, 100 + acc);
-                    break;
-                }
-                ptx::tc_fence_after();
-                int nchunks = 0;
-                if (n_valid) {
-                    const int64_t left = p.M - m0;         // > 0
-                    nchunks = left >= block_t ? chunks : (int)((left + kChunkT - 1) / kChunkT);
-                }
-                const uint32_t tbase =
-                    tmem_base + ((uint32_t)(quarter * 32 + half * 16) << 16) + (uint32_t)(acc * kAccStride);
-
-                auto release = [&]() {
-                    ptx::tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) ptx::mbar_arrive_cluster(tmem_empty);
-                };
-                // one chunk: v holds it (load issued earlier), vn receives this warp's next one
-                auto step = [&](uint32_t(&v)[16], uint32_t(&vn)[16], int c) {
-                    ptx::tmem_ld_wait_regs(v);
-                    if (c + 2 < nchunks)
-                        ptx::tmem_ld_16x256b_x4(tbase + (uint32_t)((c + 2) * kChunkT), vn);
-                    else
-                        release();                                     // all this warp reads of the tile is in registers
-                    uint32_t pk[8];
-#pragma unroll
-                    for (int i = 0; i < 4; ++i)
-#pragma unroll
-                        for (int j = 0; j < 2; ++j) {
-                            float2 y = __ffma2_rn(make_float2(__int2float_rn((int32_t)v[4 * i + 2 * j]),
-                                                              __int2float_rn((int32_t)v[4 * i + 2 * j + 1])),
-                                                  make_float2(sc[j], sc[j]), make_float2(bi[j], bi[j]));
-                            if (p.act == GPUSQ_ACT_GELU) y = gelu_pair(y);
-                            const __half2 hh = __floats2half2_rn(y.x, y.y);   // low = token 2(t%4), high = +1
-                            pk[2 * i + j] = *reinterpret_cast<const uint32_t *>(&hh);
-                        }
-                    // the staging tile's previous contents have been stored
-                    const uint32_t b = filled % kEpiBufs;
-                    if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->stg_free[group][b]),
-                                                ((filled / kEpiBufs) & 1u) ^ 1u, abort_flag, to)) {
-                        if (to && lane == 0) report_timeout(p, ctl, tile, 2, 200 + (int)b);
-                        ok = false;
-                        return;
-                    }
-                    // matrices of one stmatrix: (tokens 0-7, feat 0-7), (0-7, 8-15), (8-15, 0-7), (8-15, 8-15)
-                    const uint32_t stage = stage0 + b * kEpiBufBytes;
-                    const int mid = lane >> 3, r = lane & 7;
-#pragma unroll
-                    for (int s2 = 0; s2 < 2; ++s2) {
-                        const int tok = 16 * s2 + 8 * (mid >> 1) + r;
-                        const int c16 = chunk16 + (mid & 1);
-                        const uint32_t addr = stage + (uint32_t)(tok * 128 + ((c16 ^ (tok & 7)) << 4));
-                        ptx::stmatrix_x4_trans(addr, pk[4 * s2 + 0], pk[4 * s2 + 1], pk[4 * s2 + 2], pk[4 * s2 + 3]);
-                    }
-                    ptx::fence_proxy_async_smem();                     // this lane's writes, for the TMA store
-                    __syncwarp();
-                    if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctl->stg_full[group][b]));
-                    ++filled;
-                };
-
-                // this warp's chunks of the tile: c0, c0 + 2, ...; the two parity groups swap every tile
-                const int c0 = (par + local) & 1;
-                if (c0 >= nchunks) {
-                    release();
-                } else {
-                    uint32_t v0[16], v1[16];
-                    ptx::tmem_ld_16x256b_x4(tbase + (uint32_t)(c0 * kChunkT), v0);
-                    for (int c = c0; ok && c < nchunks; c += 4) {
-                        step(v0, v1, c);
-                        if (ok && c + 2 < nchunks) step(v1, v0, c + 2);
-                    }
-                }
-            }
+            EpiF16 e;
+            e.p = &p;
+            e.ctl = ctl;
+            e.tmem_base = tmem_base;
+            e.stage0 = stage0;
+            e.stg_full0 = ptx::smem_u32(&ctl->stg_full[group][0]);
+            e.stg_free0 = ptx::smem_u32(&ctl->stg_free[group][0]);
+            e.tmem_empty0 = tmem_empty0;
+            e.tmem_empty1 = tmem_empty1;
+            e.x_scale = x_scale;
+            e.warp = warp;
+            e.lane = lane;
+            e.rank = (int)rank;
+            e.cluster_id = cluster_id;
+            e.num_clusters = num_clusters;
+            e.tiles_n = tiles_n;
+            e.num_tiles = num_tiles;
+            e.block_t = block_t;
+            if (p.act == GPUSQ_ACT_GELU)
+                e.template run<true>();
+            else
+                e.template run<false>();
         } else {
             for (int tile = cluster_id; tile < num_tiles; tile += num_clusters, ++local) {
                 const int tn = tile % tiles_n, tm = tile / tiles_n;

@@ -56,43 +56,50 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t byt
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
                  : "memory");
 }
-// One try: the hardware parks the thread until the phase completes or about `kSuspendNs` have passed,
-// so a waiting warp issues an instruction every microsecond or so instead of competing for issue
-// slots with the warps that have work (a dozen polling warps otherwise take half of an SM's slots).
-constexpr uint32_t kSuspendNs = 1000;
+// One try: the hardware parks the thread for a short, implementation-defined time unless the
+// phase has completed.
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 {
     uint32_t ok;
     asm volatile(
         "{\n"
         ".reg .pred P;\n"
-        "mbarrier.try_wait.parity.shared::cta.b64 P, [%1], %2, %3;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 P, [%1], %2;\n"
         "selp.u32 %0, 1, 0, P;\n"
         "}\n"
         : "=r"(ok)
-        : "r"(bar), "r"(parity), "r"(kSuspendNs)
+        : "r"(bar), "r"(parity)
         : "memory");
     return ok != 0;
 }
 
 // Bounded wait: gives up after `kWaitLimitNs` of wall time, or as soon as another
 // thread of the CTA has raised *abort_flag.  Returns false on either; the
-// caller that timed out raises the flag itself.
+// caller that timed out raises the flag itself.  The common case (the phase
+// is complete already) costs one try and one branch; the retry loop is kept
+// out of line so that it does not bloat the callers' instruction streams, and
+// looks at the flag and the clock only every 32 tries.
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s
+// returns 0 = phase complete, 1 = abort flag seen, 2 = time limit reached
+__device__ __noinline__ int mbar_wait_slow(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag)
+{
+    const uint64_t t0 = globaltimer_ns();
+    for (;;) {
+#pragma unroll 1
+        for (int it = 0; it < 32; ++it)
+            if (mbar_try_wait(bar, parity)) return 0;
+        if (*abort_flag) return 1;
+        if (globaltimer_ns() - t0 > kWaitLimitNs) return 2;
+    }
+}
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
                                                   volatile uint32_t *abort_flag, bool &timed_out)
 {
     timed_out = false;
     if (mbar_try_wait(bar, parity)) return true;
-    const uint64_t t0 = globaltimer_ns();
-    for (;;) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if (globaltimer_ns() - t0 > kWaitLimitNs) {
-            timed_out = true;
-            return false;
-        }
-    }
+    const int r = mbar_wait_slow(bar, parity, abort_flag);
+    timed_out = r == 2;
+    return r == 0;
 }
 
 // ---- TMA ----
