@@ -542,8 +542,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     } else {
         // ------------------------------------------------------------ epilogue
         const int quarter = warp & 3;                      // tensor-memory lanes [32q, 32q+32) are this warp's to read
-        const int half = ((warp - 2) >> 2) & 1;            // which 16 of them (F16 path)
-        const int par = (warp - 2) >> 3;                   // which chunks: every other one
+        const int par = (warp - 2) >> 3;                   // FP16 path: which chunks, every other one
         const float x_scale = (p.out_type == GPUSQ_OUT_I32) ? 1.0f : __ldg(p.x_scale);
         const float out_scale = (p.out_type == GPUSQ_OUT_I8) ? __ldg(p.out_scale) : 1.0f;
         // the accumulators of both CTAs are released on CTA 0's barrier, where the MMA issuer waits
