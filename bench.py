@@ -229,7 +229,7 @@ def run_gpusq(args, cfg):
         state.append(dict(L=L, X=X, bias=bias, Wq=Wq, ws=ws, Wpk=Wpk,
                           Xq=torch.empty((M, L.K), dtype=torch.int8, device=dev),
                           xs=torch.empty((1,), dtype=torch.float32, device=dev),
-                          wsb=torch.empty((B.quant_act_workspace(M, L.K),), dtype=torch.uint8, device=dev),
+                          wsb=torch.zeros((B.quant_act_workspace(M, L.K),), dtype=torch.uint8, device=dev),
                           Y=torch.empty((M, L.N), dtype=torch.float16, device=dev)))
     status = torch.zeros(4, dtype=torch.int32, device=dev)
 

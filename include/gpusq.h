@@ -122,7 +122,14 @@ int gpusq_pack24(const int8_t *vals, const uint8_t *meta, void *Wpacked, int N, 
  *   Xq = clamp(round-half-even(float(X) / *x_scale), -127, 127).
  *   workspace: device scratch of at least gpusq_quant_act_workspace(M, K)
  *     bytes, 16-byte aligned, needed for GPUSQ_SCALE_COMPUTE only (may be NULL
- *     otherwise); its contents on entry do not matter.
+ *     otherwise).  It must be ZERO-FILLED before its first use (once, e.g.
+ *     right after allocation); every call leaves it usable by the next call,
+ *     of any size, so one buffer serves a whole stream of calls.  Calls that
+ *     can overlap on the GPU need separate workspaces.
+ *   GPUSQ_SCALE_COMPUTE runs as one cooperative launch whose CTAs meet at a
+ *   grid-wide barrier; its wait is bounded: if it ever expires nothing is
+ *   quantised, *x_scale is set to NaN and the workspace must be zero-filled
+ *   again.
  * Requires M > 0, K > 0, K % 8 == 0, X and Xq 16-byte aligned.
  */
 size_t gpusq_quant_act_workspace(int64_t M, int K);

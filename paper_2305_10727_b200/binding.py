@@ -167,7 +167,7 @@ def quant_act(X: torch.Tensor, Xq: Optional[torch.Tensor] = None, x_scale: Optio
             raise ValueError("scale_mode GIVEN needs x_scale")
         x_scale = torch.empty((1,), dtype=torch.float32, device=X.device)
     if workspace is None and scale_mode == SCALE_COMPUTE:
-        workspace = torch.empty((quant_act_workspace(M, K),), dtype=torch.uint8, device=X.device)
+        workspace = torch.zeros((quant_act_workspace(M, K),), dtype=torch.uint8, device=X.device)
     ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
     _check(load().gpusq_quant_act(_ptr(X), _ptr(Xq), _ptr(x_scale), scale_mode, M, K, _ptr(workspace),
                                   ws_bytes, _stream()), "gpusq_quant_act")

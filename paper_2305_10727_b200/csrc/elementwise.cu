@@ -240,7 +240,8 @@ pack24_kernel(const int8_t *__restrict__ vals, const uint8_t *__restrict__ meta,
 }
 
 // --------------------------------------------------------------- quant_act
-constexpr int kMaxPartials = 2048;   // workspace: one 32-bit partial maximum per block
+constexpr int kMaxPartials = 2048;   // workspace: one 32-bit partial maximum per block ...
+constexpr int kWorkspaceExtra = 64;  // ... and, behind them, the two counters of the grid-wide barrier
 
 __device__ __forceinline__ uint32_t absmax_bits8(uint4 v)
 {
@@ -269,34 +270,77 @@ act_absmax_kernel(const uint4 *__restrict__ X, uint32_t *__restrict__ partial, i
     if (threadIdx.x == 0) partial[blockIdx.x] = (uint32_t)r;
 }
 
-// Same code as quant_code(x, s) without the division: r = x * (1/s) is within 2^-22 |r| of the
-// exactly rounded quotient, so unless r lies within 1e-4 of a rounding boundary (k + 0.5) both
-// round to the same integer; the rare boundary case repeats the step with the true division.
-// (|r| >= 256 saturates to +-127 either way.)
-__device__ __forceinline__ int quant_code_mul(float x, float s, float inv_s)
+// clamp(round-half-even(x / s), -127, 127) for four binary16 values, packed as four INT8 codes,
+// without the division and without the conversion unit.
+//   Rounding: adding 1.5 * 2^23 in binary32 rounds to an integer with ties to even and leaves that
+//   integer, as a two's-complement byte, in the low byte of the sum's bit pattern; as the addend of
+//   a fused multiply-add it rounds the exact product x * c once.
+//   Exactness: with c_lo < 1/s < c_hi (1/s perturbed by -+2^-21, far more than its own rounding
+//   error and than the rounding error of the binary32 quotient), x/s and its binary32 rounding both
+//   lie between x * c_lo and x * c_hi; rounding is monotonic, so if both products round to the same
+//   integer, that integer is the code of the true quotient.  Otherwise (the quotient is within
+//   ~1e-4 of k + 0.5), and when 1/s is not finite, the true division decides.
+//   Clamping (kClamp, for a scale that was supplied): x is clamped to +-127 s beforehand, which
+//   gives the same code because rounding is monotonic and the bounds are integers.  A scale
+//   derived from the tensor's own maximum needs none (|x/s| <= 127 by construction).
+constexpr float kRoundMagic = 12582912.0f;     // 1.5 * 2^23
+
+struct ActScale {
+    float s;            // the scale
+    float2 c_lo, c_hi;  // the bracketing reciprocals, duplicated for packed math
+    float x_max;        // 127 s (kClamp)
+    bool always_divide; // 1/s is not finite
+};
+
+__device__ __forceinline__ ActScale make_act_scale(float s)
 {
-    float r = x * inv_s;
-    const float d = fabsf(r - rintf(r));
-    if (d > 0.5f - 1e-4f && fabsf(r) < 256.0f) r = __fdiv_rn(x, s);
-    return __float2int_rn(r);
+    ActScale a;
+    a.s = s;
+    const float inv_s = __frcp_rn(s);
+    const float lo = __fmul_rn(inv_s, 1.0f - 4.76837158203125e-7f), hi = __fmul_rn(inv_s, 1.0f + 4.76837158203125e-7f);
+    a.c_lo = make_float2(lo, lo);
+    a.c_hi = make_float2(hi, hi);
+    a.x_max = __fmul_rn(s, 127.0f);
+    a.always_divide = !(fabsf(inv_s) < 3.0e38f) || !(a.x_max < 3.0e38f);
+    return a;
 }
 
-__device__ __forceinline__ uint32_t pack4_s8_clamp127(int a, int b, int c, int d)
+template <bool kClamp>
+__device__ __forceinline__ float quant_exact_sum(float x, float s)
 {
-    // cvt.pack.sat.s8.s32.b32 r, x, y, z  gives  r = (z << 16) | (sat8(x) << 8) | sat8(y)
-    uint32_t hi, out;
-    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(d), "r"(c), "r"(0));
-    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(out) : "r"(b), "r"(a), "r"(hi));
-    return __vmaxs4(out, 0x81818181u);     // -128 -> -127
+    float r = __fdiv_rn(x, s);
+    if (kClamp) r = fminf(fmaxf(r, -127.0f), 127.0f);
+    return r + kRoundMagic;
 }
 
-__device__ __forceinline__ uint32_t quant4_f16(uint32_t lo, uint32_t hi, float s, float inv_s)
+template <bool kClamp>
+__device__ __forceinline__ uint32_t quant4_f16(uint32_t lo, uint32_t hi, const ActScale &a)
 {
-    const __half2 a = *reinterpret_cast<const __half2 *>(&lo);
-    const __half2 b = *reinterpret_cast<const __half2 *>(&hi);
-    const float2 fa = __half22float2(a), fb = __half22float2(b);
-    return pack4_s8_clamp127(quant_code_mul(fa.x, s, inv_s), quant_code_mul(fa.y, s, inv_s),
-                             quant_code_mul(fb.x, s, inv_s), quant_code_mul(fb.y, s, inv_s));
+    const float2 xa = __half22float2(*reinterpret_cast<const __half2 *>(&lo));
+    const float2 xb = __half22float2(*reinterpret_cast<const __half2 *>(&hi));
+    float2 fa = xa, fb = xb;
+    if (kClamp) {
+        fa = make_float2(fminf(fmaxf(fa.x, -a.x_max), a.x_max), fminf(fmaxf(fa.y, -a.x_max), a.x_max));
+        fb = make_float2(fminf(fmaxf(fb.x, -a.x_max), a.x_max), fminf(fmaxf(fb.y, -a.x_max), a.x_max));
+    }
+    const float2 magic = make_float2(kRoundMagic, kRoundMagic);
+    float2 ma = __ffma2_rn(fa, a.c_lo, magic), mb = __ffma2_rn(fb, a.c_lo, magic);
+    const float2 ha = __ffma2_rn(fa, a.c_hi, magic), hb = __ffma2_rn(fb, a.c_hi, magic);
+    const uint32_t differ = (__float_as_uint(ma.x) ^ __float_as_uint(ha.x)) | (__float_as_uint(ma.y) ^ __float_as_uint(ha.y)) |
+                            (__float_as_uint(mb.x) ^ __float_as_uint(hb.x)) | (__float_as_uint(mb.y) ^ __float_as_uint(hb.y));
+    if (differ != 0u || a.always_divide) {
+        ma = make_float2(quant_exact_sum<kClamp>(xa.x, a.s), quant_exact_sum<kClamp>(xa.y, a.s));
+        mb = make_float2(quant_exact_sum<kClamp>(xb.x, a.s), quant_exact_sum<kClamp>(xb.y, a.s));
+    }
+    const uint32_t p01 = __byte_perm(__float_as_uint(ma.x), __float_as_uint(ma.y), 0x0040);
+    const uint32_t p23 = __byte_perm(__float_as_uint(mb.x), __float_as_uint(mb.y), 0x0040);
+    return __byte_perm(p01, p23, 0x5410);
+}
+
+template <bool kClamp>
+__device__ __forceinline__ uint2 quant8_f16(uint4 v, const ActScale &a)
+{
+    return make_uint2(quant4_f16<kClamp>(v.x, v.y, a), quant4_f16<kClamp>(v.z, v.w, a));
 }
 
 // n_partials > 0: the scale is derived from the partial maxima and written to
@@ -317,17 +361,108 @@ act_quant_kernel(const uint4 *__restrict__ X, uint2 *__restrict__ Xq, float *x_s
     } else {
         s = *x_scale;
     }
-    const float inv_s = __frcp_rn(s);
+    const ActScale a = make_act_scale(s);
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     for (; i + stride < vec8; i += 2 * stride) {
         const uint4 v0 = __ldg(X + i), v1 = __ldg(X + i + stride);
-        Xq[i] = make_uint2(quant4_f16(v0.x, v0.y, s, inv_s), quant4_f16(v0.z, v0.w, s, inv_s));
-        Xq[i + stride] = make_uint2(quant4_f16(v1.x, v1.y, s, inv_s), quant4_f16(v1.z, v1.w, s, inv_s));
+        Xq[i] = quant8_f16<true>(v0, a);
+        Xq[i + stride] = quant8_f16<true>(v1, a);
     }
-    for (; i < vec8; i += stride) {
-        const uint4 v = __ldg(X + i);
-        Xq[i] = make_uint2(quant4_f16(v.x, v.y, s, inv_s), quant4_f16(v.z, v.w, s, inv_s));
+    for (; i < vec8; i += stride) Xq[i] = quant8_f16<true>(__ldg(X + i), a);
+}
+
+// ---- one-launch activation quantisation (scale computed from the tensor) ----
+// A cooperative grid of one 1024-thread CTA per SM.  Each CTA owns a contiguous slice of X:
+//   1. reads it once from HBM, keeps as much of it as fits in shared memory, finds max|x|;
+//   2. publishes its maximum, crosses a grid-wide barrier (two counters in the workspace, zero
+//      before and after every call; the wait is bounded) and reduces all maxima to the scale;
+//   3. quantises the slice, from shared memory where it was kept, and writes the codes.
+// So X crosses HBM once when a slice fits (up to ~200 KB per SM, 29 MB per tensor) and there is
+// one launch instead of two.  If the barrier wait expires nothing is quantised and *x_scale = NaN.
+constexpr int kFusedThreads = 1024;
+constexpr int kFusedCacheVecs = 12800;                           // 16-byte vectors kept per CTA (200 KB)
+constexpr int kFusedSmemBytes = kFusedCacheVecs * 16;
+constexpr uint64_t kGridWaitLimitNs = 2000000000ull;             // 2 s
+
+__device__ __forceinline__ uint64_t globaltimer_now()
+{
+    uint64_t t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+
+__global__ void __launch_bounds__(kFusedThreads, 1)
+act_quant_fused_kernel(const uint4 *__restrict__ X, uint2 *__restrict__ Xq, float *x_scale,
+                       uint32_t *partial, uint32_t *counters, int64_t vec8)
+{
+    extern __shared__ uint4 cache[];
+    __shared__ float red[kFusedThreads / 32];
+    __shared__ uint32_t barrier_ok;
+    const int64_t per = (vec8 + gridDim.x - 1) / gridDim.x;
+    const int64_t lo = (int64_t)blockIdx.x * per;
+    const int64_t hi = lo + per < vec8 ? lo + per : vec8;
+    const int tid = threadIdx.x;
+
+    // 1. maximum of the slice; the first kFusedCacheVecs vectors stay in shared memory
+    uint32_t m = 0;
+    int64_t i = lo + tid;
+    for (; i + 3 * kFusedThreads < hi; i += 4 * kFusedThreads) {
+        uint4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) v[u] = __ldcs(X + i + u * kFusedThreads);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            m = max(m, absmax_bits8(v[u]));
+            const int64_t idx = i + u * kFusedThreads - lo;
+            if (idx < kFusedCacheVecs) cache[idx] = v[u];
+        }
+    }
+    for (; i < hi; i += kFusedThreads) {
+        const uint4 v = __ldcs(X + i);
+        m = max(m, absmax_bits8(v));
+        if (i - lo < kFusedCacheVecs) cache[i - lo] = v;
+    }
+    const uint32_t mine = (uint32_t)block_max((float)m, red);
+
+    // 2. grid-wide maximum.  counters[0] counts arrivals, counters[1] CTAs that have seen all arrive;
+    // the last of those puts both back to zero, the state the next call on this workspace expects.
+    if (tid == 0) {
+        partial[blockIdx.x] = mine;
+        __threadfence();
+        atomicAdd(counters, 1u);
+        const uint64_t t0 = globaltimer_now();
+        uint32_t ok = 1;
+        for (uint32_t it = 1; *reinterpret_cast<volatile uint32_t *>(counters) < gridDim.x; ++it) {
+            if ((it & 255u) == 0u && globaltimer_now() - t0 > kGridWaitLimitNs) {
+                ok = 0;
+                break;
+            }
+        }
+        __threadfence();
+        if (ok && atomicAdd(counters + 1, 1u) == gridDim.x - 1) {
+            counters[0] = 0;
+            counters[1] = 0;
+        }
+        barrier_ok = ok;
+    }
+    __syncthreads();
+    if (!barrier_ok) {
+        if (blockIdx.x == 0 && tid == 0) *x_scale = __int_as_float(0x7FC00000);
+        return;
+    }
+    uint32_t g = 0;
+    for (int b = tid; b < (int)gridDim.x; b += kFusedThreads) g = max(g, __ldcg(partial + b));
+    const uint32_t bits = (uint32_t)block_max((float)g, red);
+    const float s = scale_from_amax(__half2float(__ushort_as_half((unsigned short)bits)));
+    if (blockIdx.x == 0 && tid == 0) *x_scale = s;
+    const ActScale a = make_act_scale(s);
+
+    // 3. quantise the slice
+    for (i = lo + tid; i < hi; i += kFusedThreads) {
+        const int64_t idx = i - lo;
+        const uint4 v = idx < kFusedCacheVecs ? cache[idx] : __ldg(X + i);
+        __stcs(Xq + i, quant8_f16<false>(v, a));
     }
 }
 
@@ -446,7 +581,7 @@ size_t gpusq_quant_act_workspace(int64_t M, int K)
 {
     (void)M;
     (void)K;
-    return (size_t)kMaxPartials * sizeof(uint32_t);
+    return (size_t)(kMaxPartials + kWorkspaceExtra) * sizeof(uint32_t);
 }
 
 int gpusq_quant_act(const void *X, int8_t *Xq, float *x_scale, int scale_mode, int64_t M, int K,
@@ -463,17 +598,37 @@ int gpusq_quant_act(const void *X, int8_t *Xq, float *x_scale, int scale_mode, i
     if (int st = check_arch()) return st;
     const int64_t vec8 = M * (int64_t)K / 8;
     cudaStream_t s = (cudaStream_t)stream;
-    int n_partials = 0;
     if (scale_mode == GPUSQ_SCALE_COMPUTE) {
-        n_partials = grid_for(ceil_div(vec8, 4), 8);
-        if (n_partials > kMaxPartials) n_partials = kMaxPartials;
-        act_absmax_kernel<<<n_partials, kThreads, 0, s>>>(reinterpret_cast<const uint4 *>(X),
-                                                         reinterpret_cast<uint32_t *>(workspace), vec8);
-        if (int st = launch_status()) return st;
+        // one cooperative launch: every CTA must be resident for the grid-wide barrier
+        static std::once_flag once;
+        static cudaError_t attr_err = cudaSuccess;
+        std::call_once(once, [] {
+            attr_err = cudaFuncSetAttribute(act_quant_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            kFusedSmemBytes);
+        });
+        if (attr_err != cudaSuccess) return GPUSQ_ERR_CUDA;
+        int per_sm = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, act_quant_fused_kernel, kFusedThreads,
+                                                          kFusedSmemBytes) != cudaSuccess || per_sm < 1)
+            return GPUSQ_ERR_CUDA;
+        int grid = num_sms();
+        if (grid > kMaxPartials) grid = kMaxPartials;
+        if ((int64_t)grid > vec8) grid = (int)vec8;
+        uint32_t *partial = reinterpret_cast<uint32_t *>(workspace);
+        uint32_t *counters = partial + kMaxPartials;
+        const uint4 *Xv = reinterpret_cast<const uint4 *>(X);
+        uint2 *Xqv = reinterpret_cast<uint2 *>(Xq);
+        int64_t n = vec8;
+        void *args[] = {&Xv, &Xqv, &x_scale, &partial, &counters, &n};
+        if (cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(act_quant_fused_kernel), dim3(grid),
+                                        dim3(kFusedThreads), args, kFusedSmemBytes, s) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return GPUSQ_ERR_CUDA;
+        }
+        return GPUSQ_OK;
     }
     act_quant_kernel<<<grid_for(ceil_div(vec8, 2), 8), kThreads, 0, s>>>(
-        reinterpret_cast<const uint4 *>(X), reinterpret_cast<uint2 *>(Xq), x_scale,
-        reinterpret_cast<const uint32_t *>(workspace), n_partials, vec8);
+        reinterpret_cast<const uint4 *>(X), reinterpret_cast<uint2 *>(Xq), x_scale, nullptr, 0, vec8);
     return launch_status();
 }
 
