@@ -241,7 +241,7 @@ pack24_kernel(const int8_t *__restrict__ vals, const uint8_t *__restrict__ meta,
 
 // --------------------------------------------------------------- quant_act
 constexpr int kMaxPartials = 2048;   // workspace: one 32-bit partial maximum per block ...
-constexpr int kWorkspaceExtra = 64;  // ... and, behind them, the two counters of the grid-wide barrier
+constexpr int kWorkspaceExtra = 64;  // ... and, behind them, the words of the grid-wide barrier (8-byte aligned)
 
 __device__ __forceinline__ uint32_t absmax_bits8(uint4 v)
 {
@@ -375,8 +375,8 @@ act_quant_kernel(const uint4 *__restrict__ X, uint2 *__restrict__ Xq, float *x_s
 // ---- one-launch activation quantisation (scale computed from the tensor) ----
 // A cooperative grid of one 1024-thread CTA per SM.  Each CTA owns a contiguous slice of X:
 //   1. reads it once from HBM, keeps as much of it as fits in shared memory, finds max|x|;
-//   2. publishes its maximum, crosses a grid-wide barrier (two counters in the workspace, zero
-//      before and after every call; the wait is bounded) and reduces all maxima to the scale;
+//   2. merges its maximum into a global one and crosses a grid-wide barrier (three words in the
+//      workspace, zero before and after every call; the wait is bounded);
 //   3. quantises the slice, from shared memory where it was kept, and writes the codes.
 // So X crosses HBM once when a slice fits (up to ~200 KB per SM, 29 MB per tensor) and there is
 // one launch instead of two.  If the barrier wait expires nothing is quantised and *x_scale = NaN.
@@ -394,11 +394,11 @@ __device__ __forceinline__ uint64_t globaltimer_now()
 
 __global__ void __launch_bounds__(kFusedThreads, 1)
 act_quant_fused_kernel(const uint4 *__restrict__ X, uint2 *__restrict__ Xq, float *x_scale,
-                       uint32_t *partial, uint32_t *counters, int64_t vec8)
+                       uint32_t *counters, int64_t vec8)
 {
     extern __shared__ uint4 cache[];
     __shared__ float red[kFusedThreads / 32];
-    __shared__ uint32_t barrier_ok;
+    __shared__ uint32_t barrier_ok, grid_max_bits;
     const int64_t per = (vec8 + gridDim.x - 1) / gridDim.x;
     const int64_t lo = (int64_t)blockIdx.x * per;
     const int64_t hi = lo + per < vec8 ? lo + per : vec8;
@@ -410,7 +410,11 @@ act_quant_fused_kernel(const uint4 *__restrict__ X, uint2 *__restrict__ Xq, floa
     for (; i + 3 * kFusedThreads < hi; i += 4 * kFusedThreads) {
         uint4 v[4];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) v[u] = __ldcs(X + i + u * kFusedThreads);
+        for (int u = 0; u < 4; ++u) {
+            // what is kept in shared memory is not needed again; the rest is re-read in step 3: leave it in L2
+            const int64_t j = i + u * kFusedThreads;
+            v[u] = j - lo < kFusedCacheVecs ? __ldcs(X + j) : __ldg(X + j);
+        }
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             m = max(m, absmax_bits8(v[u]));
@@ -419,42 +423,44 @@ act_quant_fused_kernel(const uint4 *__restrict__ X, uint2 *__restrict__ Xq, floa
         }
     }
     for (; i < hi; i += kFusedThreads) {
-        const uint4 v = __ldcs(X + i);
+        const uint4 v = i - lo < kFusedCacheVecs ? __ldcs(X + i) : __ldg(X + i);
         m = max(m, absmax_bits8(v));
         if (i - lo < kFusedCacheVecs) cache[i - lo] = v;
     }
     const uint32_t mine = (uint32_t)block_max((float)m, red);
 
-    // 2. grid-wide maximum.  counters[0] counts arrivals, counters[1] CTAs that have seen all arrive;
-    // the last of those puts both back to zero, the state the next call on this workspace expects.
+    // 2. grid-wide maximum.  One 8-byte word holds {arrivals, maximum}: a CTA first merges its maximum,
+    // then counts itself in, so a single 8-byte read that sees every arrival also sees the final
+    // maximum.  counters[2] counts the CTAs that have read it; the last of them puts all three words
+    // back to zero, the state the next call on this workspace expects.
     if (tid == 0) {
-        partial[blockIdx.x] = mine;
+        atomicMax(counters + 1, mine);
         __threadfence();
         atomicAdd(counters, 1u);
         const uint64_t t0 = globaltimer_now();
         uint32_t ok = 1;
-        for (uint32_t it = 1; *reinterpret_cast<volatile uint32_t *>(counters) < gridDim.x; ++it) {
+        uint2 word;
+        for (uint32_t it = 1;; ++it) {
+            word = __ldcv(reinterpret_cast<const uint2 *>(counters));
+            if (word.x >= gridDim.x) break;
             if ((it & 255u) == 0u && globaltimer_now() - t0 > kGridWaitLimitNs) {
                 ok = 0;
                 break;
             }
         }
-        __threadfence();
-        if (ok && atomicAdd(counters + 1, 1u) == gridDim.x - 1) {
-            counters[0] = 0;
-            counters[1] = 0;
+        if (ok && atomicAdd(counters + 2, 1u) == gridDim.x - 1) {
+            __stcg(reinterpret_cast<uint2 *>(counters), make_uint2(0u, 0u));
+            counters[2] = 0;
         }
         barrier_ok = ok;
+        grid_max_bits = word.y;
     }
     __syncthreads();
     if (!barrier_ok) {
         if (blockIdx.x == 0 && tid == 0) *x_scale = __int_as_float(0x7FC00000);
         return;
     }
-    uint32_t g = 0;
-    for (int b = tid; b < (int)gridDim.x; b += kFusedThreads) g = max(g, __ldcg(partial + b));
-    const uint32_t bits = (uint32_t)block_max((float)g, red);
-    const float s = scale_from_amax(__half2float(__ushort_as_half((unsigned short)bits)));
+    const float s = scale_from_amax(__half2float(__ushort_as_half((unsigned short)grid_max_bits)));
     if (blockIdx.x == 0 && tid == 0) *x_scale = s;
     const ActScale a = make_act_scale(s);
 
@@ -614,12 +620,11 @@ int gpusq_quant_act(const void *X, int8_t *Xq, float *x_scale, int scale_mode, i
         int grid = num_sms();
         if (grid > kMaxPartials) grid = kMaxPartials;
         if ((int64_t)grid > vec8) grid = (int)vec8;
-        uint32_t *partial = reinterpret_cast<uint32_t *>(workspace);
-        uint32_t *counters = partial + kMaxPartials;
+        uint32_t *counters = reinterpret_cast<uint32_t *>(workspace) + kMaxPartials;
         const uint4 *Xv = reinterpret_cast<const uint4 *>(X);
         uint2 *Xqv = reinterpret_cast<uint2 *>(Xq);
         int64_t n = vec8;
-        void *args[] = {&Xv, &Xqv, &x_scale, &partial, &counters, &n};
+        void *args[] = {&Xv, &Xqv, &x_scale, &counters, &n};
         if (cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(act_quant_fused_kernel), dim3(grid),
                                         dim3(kFusedThreads), args, kFusedSmemBytes, s) != cudaSuccess) {
             (void)cudaGetLastError();
