@@ -403,6 +403,8 @@ act_quant_fused_kernel(const uint4 *__restrict__ X, uint2 *__restrict__ Xq, floa
     const int64_t lo = (int64_t)blockIdx.x * per;
     const int64_t hi = lo + per < vec8 ? lo + per : vec8;
     const int tid = threadIdx.x;
+    // the next kernel of the stream may be scheduled as soon as CTAs of this grid make room
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     // 1. maximum of the slice; the first kFusedCacheVecs vectors stay in shared memory
     uint32_t m = 0;

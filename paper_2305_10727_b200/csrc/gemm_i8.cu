@@ -386,6 +386,11 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     ptx::cluster_sync();            // the other CTA's barriers exist before anything is signalled on them
     ptx::tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
+    // Programmatic dependent launch: everything above ran while the previous kernel in the stream was
+    // still finishing; its results (activations, their scale) may be read from here on.  The next
+    // kernel in the stream may start its own set-up now.
+    ptx::grid_dependency_wait();
+    ptx::grid_launch_dependents();
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer
@@ -798,8 +803,21 @@ static int launch_gemm(const int8_t *Xq, const void *Wsrc, const float *w_scale,
 
     const int64_t tiles = (int64_t)tiles_n * ceil_div(M, block_t);
     const int grid = 2 * (int)(tiles < clusters ? tiles : clusters);
-    gemm_i8_kernel<kSparse><<<grid, kNumThreads, C::kSmemBytes, (cudaStream_t)stream>>>(map_a, map_b, map_e, map_y, p);
-    return launch_status();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid, 1, 1);
+    cfg.blockDim = dim3(kNumThreads, 1, 1);
+    cfg.dynamicSmemBytes = C::kSmemBytes;
+    cfg.stream = (cudaStream_t)stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;     // start while the previous kernel drains
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, gemm_i8_kernel<kSparse>, map_a, map_b, map_e, map_y, p) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return GPUSQ_ERR_CUDA;
+    }
+    return GPUSQ_OK;
 }
 
 }  // namespace gpusq

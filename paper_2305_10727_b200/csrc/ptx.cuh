@@ -355,6 +355,13 @@ __device__ __forceinline__ void tmem_ld_wait_regs(uint32_t (&r)[16])
                  : "memory");
 }
 
+// ---- programmatic dependent launch ----
+// wait until the kernel this one depends on has completed and its writes are visible (returns at
+// once when the launch carried no programmatic dependency)
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// let the next kernel of the stream be scheduled as soon as this grid's CTAs make room
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---- descriptors ----
 // Shared-memory matrix descriptor for a K-major operand tile whose rows are
 // `swizzle_bytes` long (32/64/128-byte swizzle) or, with swizzle_bytes == 0,
