@@ -129,14 +129,14 @@ __device__ __forceinline__ void report_timeout(const GemmParams &p, Ctl *ctl, in
 // Exact-erf GELU as GELU(y) = max(y, 0) - g(|y|), g(t) = t * Phi(-t) = t * 2^p(t) with
 // p(t) = log2(Phi(-t)) a degree-7 polynomial on [0, 6] (gen_gelu_coeffs.py; |error| < 6e-6 in p,
 // so g keeps a relative accuracy of ~4e-6 even in the negative tail).  Beyond t = 6, g < 2^-25.
-constexpr float kGeluC0 = -9.999943376e-01f;
-constexpr float kGeluC1 = -1.151269197e+00f;
-constexpr float kGeluC2 = -4.584097862e-01f;
-constexpr float kGeluC3 = -5.402068794e-02f;
-constexpr float kGeluC4 = 8.539461531e-03f;
-constexpr float kGeluC5 = -9.388679173e-04f;
-constexpr float kGeluC6 = 6.268139987e-05f;
-constexpr float kGeluC7 = -1.889626219e-06f;
+// coefficients of p, each duplicated so that a packed FP32 instruction can take the pair straight
+// from the constant bank
+__constant__ float2 kGeluC[8] = {
+    {-9.999943376e-01f, -9.999943376e-01f}, {-1.151269197e+00f, -1.151269197e+00f},
+    {-4.584097862e-01f, -4.584097862e-01f}, {-5.402068794e-02f, -5.402068794e-02f},
+    {8.539461531e-03f, 8.539461531e-03f},   {-9.388679173e-04f, -9.388679173e-04f},
+    {6.268139987e-05f, 6.268139987e-05f},   {-1.889626219e-06f, -1.889626219e-06f},
+};
 
 __device__ __forceinline__ float ex2_approx(float x)
 {
@@ -149,16 +149,12 @@ __device__ __forceinline__ float ex2_approx(float x)
 __device__ __forceinline__ float2 gelu_pair(float2 y)
 {
     const float2 t = make_float2(fminf(fabsf(y.x), 6.0f), fminf(fabsf(y.y), 6.0f));
-    float2 r = make_float2(kGeluC7, kGeluC7);
-    r = __ffma2_rn(r, t, make_float2(kGeluC6, kGeluC6));
-    r = __ffma2_rn(r, t, make_float2(kGeluC5, kGeluC5));
-    r = __ffma2_rn(r, t, make_float2(kGeluC4, kGeluC4));
-    r = __ffma2_rn(r, t, make_float2(kGeluC3, kGeluC3));
-    r = __ffma2_rn(r, t, make_float2(kGeluC2, kGeluC2));
-    r = __ffma2_rn(r, t, make_float2(kGeluC1, kGeluC1));
-    r = __ffma2_rn(r, t, make_float2(kGeluC0, kGeluC0));
+    float2 r = kGeluC[7];
+#pragma unroll
+    for (int d = 6; d >= 0; --d) r = __ffma2_rn(r, t, kGeluC[d]);
     const float2 g = __fmul2_rn(t, make_float2(ex2_approx(r.x), ex2_approx(r.y)));
-    return make_float2(fmaxf(y.x, 0.0f) - g.x, fmaxf(y.y, 0.0f) - g.y);
+    // max(y, 0) - g
+    return __ffma2_rn(g, make_float2(-1.0f, -1.0f), make_float2(fmaxf(y.x, 0.0f), fmaxf(y.y, 0.0f)));
 }
 
 __device__ __forceinline__ float gelu_one(float y)

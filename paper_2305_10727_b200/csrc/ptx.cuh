@@ -80,14 +80,17 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 // out of line so that it does not bloat the callers' instruction streams, and
 // looks at the flag and the clock only every 32 tries.
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s
+constexpr uint32_t kRetrySleepNs = 100;
 // returns 0 = phase complete, 1 = abort flag seen, 2 = time limit reached
 __device__ __noinline__ int mbar_wait_slow(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag)
 {
     const uint64_t t0 = globaltimer_ns();
     for (;;) {
 #pragma unroll 1
-        for (int it = 0; it < 32; ++it)
+        for (int it = 0; it < 32; ++it) {
             if (mbar_try_wait(bar, parity)) return 0;
+            __nanosleep(kRetrySleepNs);          // leave the issue slots to the warps that have work
+        }
         if (*abort_flag) return 1;
         if (globaltimer_ns() - t0 > kWaitLimitNs) return 2;
     }
