@@ -36,9 +36,10 @@ UNIT = "TOPS"
 NOMINAL_SPARSE_INT8_TOPS = 9000.0      # NVIDIA's dense-half figure for B200 INT8 with 2:4 sparsity (4 x 2250 BF16)
 NOMINAL_BF16_TFLOPS = 2250.0
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# DRAM bytes per launch of the dominant kernel from the ncu capture summarised in
-# profiles/gemm_i8_sparse_deit_base_qkv.md (None until a capture exists)
-NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+# dram__bytes_read.sum + dram__bytes_write.sum of the four sparse-GEMM launches of one step, from the
+# ncu capture summarised in profiles/gemm_i8_sparse_deit_base_block.md (cold L2 per launch: most of
+# the FP16 output is still in L2 when a launch ends).  Set to None when the kernel changes.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 96.0e6
 
 
 def load_peaks():
