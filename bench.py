@@ -181,6 +181,7 @@ def run_gpusq(args, cfg):
     import torch.distributed as dist
 
     from paper_2305_10727_b200 import binding as B
+    from paper_2305_10727_b200 import replicas
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -340,13 +341,10 @@ def run_gpusq(args, cfg):
     clocks = sampler.stop()
     status_host = status.cpu().tolist()
 
-    if world > 1:
-        t = torch.tensor([ms_step], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_step = float(t.item())
+    ms_step = replicas.max_over_ranks(ms_step, dev)          # the slowest rank's time
 
     flops_step = sum(layer_flops(M, L) for L in layers)
-    value = world * flops_step / (ms_step * 1e-3) / 1e12
+    value = replicas.whole_job_throughput(flops_step, ms_step * 1e-3, world) / 1e12
 
     # ---- roofline of the dominant kernel (the sparse GEMM, all four shapes of the block)
     gemm_mean = {k: statistics.fmean(v) for k, v in gemm_us.items()}
@@ -406,10 +404,7 @@ def run_gpusq(args, cfg):
         e1.record(stream)
         barrier()
         ms_e2e = e0.elapsed_time(e1) / n_e2e
-        if world > 1:
-            t = torch.tensor([ms_e2e], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_e2e = float(t.item())
+        ms_e2e = replicas.max_over_ranks(ms_e2e, dev)
         e2e = {"value": round(world * flops_step / (ms_e2e * 1e-3) / 1e12, 2), "unit": UNIT,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": round(ms_e2e, 4), "steps": n_e2e}
 
