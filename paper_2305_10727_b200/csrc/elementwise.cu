@@ -313,34 +313,47 @@ __device__ __forceinline__ float quant_exact_sum(float x, float s)
     return r + kRoundMagic;
 }
 
+// two binary16 values -> the two sums whose low bytes are the codes; `differ` collects the bits in
+// which the bracketing products disagree
 template <bool kClamp>
-__device__ __forceinline__ uint32_t quant4_f16(uint32_t lo, uint32_t hi, const ActScale &a)
+__device__ __forceinline__ float2 quant2_sums(uint32_t h2, const ActScale &a, uint32_t &differ)
 {
-    const float2 xa = __half22float2(*reinterpret_cast<const __half2 *>(&lo));
-    const float2 xb = __half22float2(*reinterpret_cast<const __half2 *>(&hi));
-    float2 fa = xa, fb = xb;
-    if (kClamp) {
-        fa = make_float2(fminf(fmaxf(fa.x, -a.x_max), a.x_max), fminf(fmaxf(fa.y, -a.x_max), a.x_max));
-        fb = make_float2(fminf(fmaxf(fb.x, -a.x_max), a.x_max), fminf(fmaxf(fb.y, -a.x_max), a.x_max));
-    }
+    float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&h2));
+    if (kClamp) f = make_float2(fminf(fmaxf(f.x, -a.x_max), a.x_max), fminf(fmaxf(f.y, -a.x_max), a.x_max));
     const float2 magic = make_float2(kRoundMagic, kRoundMagic);
-    float2 ma = __ffma2_rn(fa, a.c_lo, magic), mb = __ffma2_rn(fb, a.c_lo, magic);
-    const float2 ha = __ffma2_rn(fa, a.c_hi, magic), hb = __ffma2_rn(fb, a.c_hi, magic);
-    const uint32_t differ = (__float_as_uint(ma.x) ^ __float_as_uint(ha.x)) | (__float_as_uint(ma.y) ^ __float_as_uint(ha.y)) |
-                            (__float_as_uint(mb.x) ^ __float_as_uint(hb.x)) | (__float_as_uint(mb.y) ^ __float_as_uint(hb.y));
-    if (differ != 0u || a.always_divide) {
-        ma = make_float2(quant_exact_sum<kClamp>(xa.x, a.s), quant_exact_sum<kClamp>(xa.y, a.s));
-        mb = make_float2(quant_exact_sum<kClamp>(xb.x, a.s), quant_exact_sum<kClamp>(xb.y, a.s));
-    }
-    const uint32_t p01 = __byte_perm(__float_as_uint(ma.x), __float_as_uint(ma.y), 0x0040);
-    const uint32_t p23 = __byte_perm(__float_as_uint(mb.x), __float_as_uint(mb.y), 0x0040);
-    return __byte_perm(p01, p23, 0x5410);
+    const float2 lo = __ffma2_rn(f, a.c_lo, magic), hi = __ffma2_rn(f, a.c_hi, magic);
+    differ |= (__float_as_uint(lo.x) ^ __float_as_uint(hi.x)) | (__float_as_uint(lo.y) ^ __float_as_uint(hi.y));
+    return lo;
 }
 
 template <bool kClamp>
+__device__ __forceinline__ float2 quant2_exact(uint32_t h2, const ActScale &a)
+{
+    const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&h2));
+    return make_float2(quant_exact_sum<kClamp>(f.x, a.s), quant_exact_sum<kClamp>(f.y, a.s));
+}
+
+__device__ __forceinline__ uint32_t pack4_low_bytes(float2 m01, float2 m23)
+{
+    const uint32_t p01 = __byte_perm(__float_as_uint(m01.x), __float_as_uint(m01.y), 0x0040);
+    const uint32_t p23 = __byte_perm(__float_as_uint(m23.x), __float_as_uint(m23.y), 0x0040);
+    return __byte_perm(p01, p23, 0x5410);
+}
+
+// eight binary16 values (16 bytes) -> eight INT8 codes (8 bytes); one exactness test for all eight
+template <bool kClamp>
 __device__ __forceinline__ uint2 quant8_f16(uint4 v, const ActScale &a)
 {
-    return make_uint2(quant4_f16<kClamp>(v.x, v.y, a), quant4_f16<kClamp>(v.z, v.w, a));
+    uint32_t differ = 0;
+    float2 m0 = quant2_sums<kClamp>(v.x, a, differ), m1 = quant2_sums<kClamp>(v.y, a, differ);
+    float2 m2 = quant2_sums<kClamp>(v.z, a, differ), m3 = quant2_sums<kClamp>(v.w, a, differ);
+    if (differ != 0u || a.always_divide) {
+        m0 = quant2_exact<kClamp>(v.x, a);
+        m1 = quant2_exact<kClamp>(v.y, a);
+        m2 = quant2_exact<kClamp>(v.z, a);
+        m3 = quant2_exact<kClamp>(v.w, a);
+    }
+    return make_uint2(pack4_low_bytes(m0, m1), pack4_low_bytes(m2, m3));
 }
 
 // n_partials > 0: the scale is derived from the partial maxima and written to
@@ -406,29 +419,39 @@ act_quant_fused_kernel(const uint4 *__restrict__ X, uint2 *__restrict__ Xq, floa
     // the next kernel of the stream may be scheduled as soon as CTAs of this grid make room
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
-    // 1. maximum of the slice; the first kFusedCacheVecs vectors stay in shared memory
+    // The slice in 32-bit terms: n vectors from Xs; the first n_kept of them stay in shared memory.
+    const int n = hi > lo ? (int)(hi - lo) : 0;             // host side: per < 2^31
+    const int n_kept = n < kFusedCacheVecs ? n : kFusedCacheVecs;
+    const uint4 *Xs = X + lo;
+    uint2 *Xqs = Xq + lo;
+
+    // 1. maximum of the slice
     uint32_t m = 0;
-    int64_t i = lo + tid;
-    for (; i + 3 * kFusedThreads < hi; i += 4 * kFusedThreads) {
+    int i = tid;
+    for (; i + 3 * kFusedThreads < n_kept; i += 4 * kFusedThreads) {
         uint4 v[4];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            // what is kept in shared memory is not needed again; the rest is re-read in step 3: leave it in L2
-            const int64_t j = i + u * kFusedThreads;
-            v[u] = j - lo < kFusedCacheVecs ? __ldcs(X + j) : __ldg(X + j);
-        }
+        for (int u = 0; u < 4; ++u) v[u] = __ldcs(Xs + i + u * kFusedThreads);   // kept: not needed from L2 again
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             m = max(m, absmax_bits8(v[u]));
-            const int64_t idx = i + u * kFusedThreads - lo;
-            if (idx < kFusedCacheVecs) cache[idx] = v[u];
+            cache[i + u * kFusedThreads] = v[u];
         }
     }
-    for (; i < hi; i += kFusedThreads) {
-        const uint4 v = i - lo < kFusedCacheVecs ? __ldcs(X + i) : __ldg(X + i);
+    for (; i < n_kept; i += kFusedThreads) {
+        const uint4 v = __ldcs(Xs + i);
         m = max(m, absmax_bits8(v));
-        if (i - lo < kFusedCacheVecs) cache[i - lo] = v;
+        cache[i] = v;
     }
+    // the rest is re-read in step 3: plain loads leave it in L2 (i continues at n_kept + its lane offset)
+    for (; i + 3 * kFusedThreads < n; i += 4 * kFusedThreads) {
+        uint4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) v[u] = __ldg(Xs + i + u * kFusedThreads);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) m = max(m, absmax_bits8(v[u]));
+    }
+    for (; i < n; i += kFusedThreads) m = max(m, absmax_bits8(__ldg(Xs + i)));
     const uint32_t mine = (uint32_t)block_max((float)m, red);
 
     // 2. grid-wide maximum.  One 8-byte word holds {arrivals, maximum}: a CTA first merges its maximum,
@@ -466,12 +489,14 @@ act_quant_fused_kernel(const uint4 *__restrict__ X, uint2 *__restrict__ Xq, floa
     if (blockIdx.x == 0 && tid == 0) *x_scale = s;
     const ActScale a = make_act_scale(s);
 
-    // 3. quantise the slice
-    for (i = lo + tid; i < hi; i += kFusedThreads) {
-        const int64_t idx = i - lo;
-        const uint4 v = idx < kFusedCacheVecs ? cache[idx] : __ldg(X + i);
-        __stcs(Xq + i, quant8_f16<false>(v, a));
+    // 3. quantise the slice: what was kept, from shared memory; the rest, from L2 / HBM
+    for (i = tid; i < n_kept; i += kFusedThreads) __stcs(Xqs + i, quant8_f16<false>(cache[i], a));
+    for (; i + kFusedThreads < n; i += 2 * kFusedThreads) {
+        const uint4 v0 = __ldg(Xs + i), v1 = __ldg(Xs + i + kFusedThreads);
+        __stcs(Xqs + i, quant8_f16<false>(v0, a));
+        __stcs(Xqs + i + kFusedThreads, quant8_f16<false>(v1, a));
     }
+    for (; i < n; i += kFusedThreads) __stcs(Xqs + i, quant8_f16<false>(__ldg(Xs + i), a));
 }
 
 // ---- library-owned scratch for gpusq_quant_act_static ----
@@ -622,6 +647,7 @@ int gpusq_quant_act(const void *X, int8_t *Xq, float *x_scale, int scale_mode, i
         int grid = num_sms();
         if (grid > kMaxPartials) grid = kMaxPartials;
         if ((int64_t)grid > vec8) grid = (int)vec8;
+        if (ceil_div(vec8, grid) > 0x7FFFFFFF) return GPUSQ_ERR_SHAPE;      // a CTA's slice is indexed with 32 bits
         uint32_t *counters = reinterpret_cast<uint32_t *>(workspace) + kMaxPartials;
         const uint4 *Xv = reinterpret_cast<const uint4 *>(X);
         uint2 *Xqv = reinterpret_cast<uint2 *>(Xq);
