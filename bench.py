@@ -387,20 +387,46 @@ def run_gpusq(args, cfg):
         h2d = sum(x.numel() * 2 for x in hX)
         d2h = sum(y.numel() * 2 for y in hY)
 
+        # Three streams, as a serving loop would run it: host -> device copies of the next layer's
+        # activations, the kernels, and device -> host copies of finished outputs overlap (the two copy
+        # directions use separate DMA engines).  Events order each layer's copy-in -> kernels -> copy-out
+        # and keep a step from overwriting buffers the previous step still uses.
+        s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+        ev_in = [torch.cuda.Event() for _ in state]
+        ev_done = [torch.cuda.Event() for _ in state]
+        ev_out = [torch.cuda.Event() for _ in state]
+        first = [True]
+
         def e2e_step():
-            for s, hx in zip(state, hX):
-                s["X"].copy_(hx, non_blocking=True)
-            run_step()
-            for s, hy in zip(state, hY):
-                hy.copy_(s["Y"], non_blocking=True)
+            for i, (s, hx, hy) in enumerate(zip(state, hX, hY)):
+                if not first[0]:
+                    s_in.wait_event(ev_done[i])          # last step's kernels have read X
+                with torch.cuda.stream(s_in):
+                    s["X"].copy_(hx, non_blocking=True)
+                    ev_in[i].record(s_in)
+                stream.wait_event(ev_in[i])
+                if not first[0]:
+                    stream.wait_event(ev_out[i])         # last step's copy-out has read Y
+                layer_quant(s)
+                layer_gemm(s)
+                ev_done[i].record(stream)
+                s_out.wait_event(ev_done[i])
+                with torch.cuda.stream(s_out):
+                    hy.copy_(s["Y"], non_blocking=True)
+                    ev_out[i].record(s_out)
+            first[0] = False
 
         for _ in range(3):
             e2e_step()
         barrier()
         n_e2e = max(3, min(args.steps, 10))
         e0.record(stream)
+        s_in.wait_event(e0)
+        s_out.wait_event(e0)
         for _ in range(n_e2e):
             e2e_step()
+        for ev in ev_out:
+            stream.wait_event(ev)
         e1.record(stream)
         barrier()
         ms_e2e = e0.elapsed_time(e1) / n_e2e
