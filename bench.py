@@ -332,6 +332,13 @@ def run_gpusq(args, cfg):
         name = s["L"].name
         gemm_us[name] = [max(ms_full - loop_ms(step_without(skip_gemm=(i,))), 1e-3) * 1e3]
         quant_us[name] = [max(ms_full - loop_ms(step_without(skip_quant=(i,))), 1e-3) * 1e3]
+    # the same step with the activation scales supplied (calibrated once, as the paper's deployed model
+    # does with its learned scales) instead of computed from every batch: extra information
+    def step_static_scale():
+        for s in state:
+            B.quant_act(s["X"], Xq=s["Xq"], x_scale=s["xs"], scale_mode=B.SCALE_GIVEN)
+            layer_gemm(s)
+    ms_static = loop_ms(step_static_scale)
     ms_dense = loop_ms(step_without(gemm=layer_gemm_dense))
     for i, s in enumerate(state):
         name = s["L"].name
@@ -464,6 +471,9 @@ def run_gpusq(args, cfg):
             "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e,
             "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
             "layers": per_layer, "prep_us": {k: round(v, 2) for k, v in prep_us.items()},
+            "static_scale_step": {"block_us": round(ms_static * 1e3, 2),
+                                  "value": round(flops_step / (ms_static * 1e-3) / 1e12, 2), "unit": UNIT,
+                                  "note": "same step with supplied activation scales (GPUSQ_SCALE_GIVEN); rank 0 only"},
             "device_status": status_host, "peaks": {k: v for k, v in peaks.items() if k in ("hbm_gbs", "bf16_tflops", "bf16_tflops_sustained", "_source")},
         }
         print(json.dumps(line))
