@@ -7,6 +7,7 @@
 #include <mutex>
 
 #include "common.cuh"
+#include "quant_math.cuh"
 
 namespace gpusq {
 
@@ -270,88 +271,21 @@ act_absmax_kernel(const uint4 *__restrict__ X, uint32_t *__restrict__ partial, i
     if (threadIdx.x == 0) partial[blockIdx.x] = (uint32_t)r;
 }
 
-// clamp(round-half-even(x / s), -127, 127) for four binary16 values, packed as four INT8 codes,
-// without the division and without the conversion unit.
-//   Rounding: adding 1.5 * 2^23 in binary32 rounds to an integer with ties to even and leaves that
-//   integer, as a two's-complement byte, in the low byte of the sum's bit pattern; as the addend of
-//   a fused multiply-add it rounds the exact product x * c once.
-//   Exactness: with c_lo < 1/s < c_hi (1/s perturbed by -+2^-21, far more than its own rounding
-//   error and than the rounding error of the binary32 quotient), x/s and its binary32 rounding both
-//   lie between x * c_lo and x * c_hi; rounding is monotonic, so if both products round to the same
-//   integer, that integer is the code of the true quotient.  Otherwise (the quotient is within
-//   ~1e-4 of k + 0.5), and when 1/s is not finite, the true division decides.
-//   Clamping (kClamp, for a scale that was supplied): x is clamped to +-127 s beforehand, which
-//   gives the same code because rounding is monotonic and the bounds are integers.  A scale
-//   derived from the tensor's own maximum needs none (|x/s| <= 127 by construction).
-constexpr float kRoundMagic = 12582912.0f;     // 1.5 * 2^23
-
-struct ActScale {
-    float s;            // the scale
-    float2 c_lo, c_hi;  // the bracketing reciprocals, duplicated for packed math
-    float x_max;        // 127 s (kClamp)
-    bool always_divide; // 1/s is not finite
-};
-
-__device__ __forceinline__ ActScale make_act_scale(float s)
-{
-    ActScale a;
-    a.s = s;
-    const float inv_s = __frcp_rn(s);
-    const float lo = __fmul_rn(inv_s, 1.0f - 4.76837158203125e-7f), hi = __fmul_rn(inv_s, 1.0f + 4.76837158203125e-7f);
-    a.c_lo = make_float2(lo, lo);
-    a.c_hi = make_float2(hi, hi);
-    a.x_max = __fmul_rn(s, 127.0f);
-    a.always_divide = !(fabsf(inv_s) < 3.0e38f) || !(a.x_max < 3.0e38f);
-    return a;
-}
-
-template <bool kClamp>
-__device__ __forceinline__ float quant_exact_sum(float x, float s)
-{
-    float r = __fdiv_rn(x, s);
-    if (kClamp) r = fminf(fmaxf(r, -127.0f), 127.0f);
-    return r + kRoundMagic;
-}
-
-// two binary16 values -> the two sums whose low bytes are the codes; `differ` collects the bits in
-// which the bracketing products disagree
-template <bool kClamp>
-__device__ __forceinline__ float2 quant2_sums(uint32_t h2, const ActScale &a, uint32_t &differ)
-{
-    float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&h2));
-    if (kClamp) f = make_float2(fminf(fmaxf(f.x, -a.x_max), a.x_max), fminf(fmaxf(f.y, -a.x_max), a.x_max));
-    const float2 magic = make_float2(kRoundMagic, kRoundMagic);
-    const float2 lo = __ffma2_rn(f, a.c_lo, magic), hi = __ffma2_rn(f, a.c_hi, magic);
-    differ |= (__float_as_uint(lo.x) ^ __float_as_uint(hi.x)) | (__float_as_uint(lo.y) ^ __float_as_uint(hi.y));
-    return lo;
-}
-
-template <bool kClamp>
-__device__ __forceinline__ float2 quant2_exact(uint32_t h2, const ActScale &a)
-{
-    const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&h2));
-    return make_float2(quant_exact_sum<kClamp>(f.x, a.s), quant_exact_sum<kClamp>(f.y, a.s));
-}
-
-__device__ __forceinline__ uint32_t pack4_low_bytes(float2 m01, float2 m23)
-{
-    const uint32_t p01 = __byte_perm(__float_as_uint(m01.x), __float_as_uint(m01.y), 0x0040);
-    const uint32_t p23 = __byte_perm(__float_as_uint(m23.x), __float_as_uint(m23.y), 0x0040);
-    return __byte_perm(p01, p23, 0x5410);
-}
-
 // eight binary16 values (16 bytes) -> eight INT8 codes (8 bytes); one exactness test for all eight
+__device__ __forceinline__ float2 h2f(uint32_t h2) { return __half22float2(*reinterpret_cast<const __half2 *>(&h2)); }
+
 template <bool kClamp>
-__device__ __forceinline__ uint2 quant8_f16(uint4 v, const ActScale &a)
+__device__ __forceinline__ uint2 quant8_f16(uint4 v, const QuantScale &a)
 {
     uint32_t differ = 0;
-    float2 m0 = quant2_sums<kClamp>(v.x, a, differ), m1 = quant2_sums<kClamp>(v.y, a, differ);
-    float2 m2 = quant2_sums<kClamp>(v.z, a, differ), m3 = quant2_sums<kClamp>(v.w, a, differ);
+    const float2 f0 = h2f(v.x), f1 = h2f(v.y), f2 = h2f(v.z), f3 = h2f(v.w);
+    float2 m0 = quant2_sums<kClamp>(f0, a, differ), m1 = quant2_sums<kClamp>(f1, a, differ);
+    float2 m2 = quant2_sums<kClamp>(f2, a, differ), m3 = quant2_sums<kClamp>(f3, a, differ);
     if (differ != 0u || a.always_divide) {
-        m0 = quant2_exact<kClamp>(v.x, a);
-        m1 = quant2_exact<kClamp>(v.y, a);
-        m2 = quant2_exact<kClamp>(v.z, a);
-        m3 = quant2_exact<kClamp>(v.w, a);
+        m0 = quant2_exact<kClamp>(f0, a);
+        m1 = quant2_exact<kClamp>(f1, a);
+        m2 = quant2_exact<kClamp>(f2, a);
+        m3 = quant2_exact<kClamp>(f3, a);
     }
     return make_uint2(pack4_low_bytes(m0, m1), pack4_low_bytes(m2, m3));
 }
@@ -374,7 +308,7 @@ act_quant_kernel(const uint4 *__restrict__ X, uint2 *__restrict__ Xq, float *x_s
     } else {
         s = *x_scale;
     }
-    const ActScale a = make_act_scale(s);
+    const QuantScale a = make_quant_scale(s);
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     for (; i + stride < vec8; i += 2 * stride) {
@@ -487,7 +421,7 @@ act_quant_fused_kernel(const uint4 *__restrict__ X, uint2 *__restrict__ Xq, floa
     }
     const float s = scale_from_amax(__half2float(__ushort_as_half((unsigned short)grid_max_bits)));
     if (blockIdx.x == 0 && tid == 0) *x_scale = s;
-    const ActScale a = make_act_scale(s);
+    const QuantScale a = make_quant_scale(s);
 
     // 3. quantise the slice: what was kept, from shared memory; the rest, from L2 / HBM
     for (i = tid; i < n_kept; i += kFusedThreads) __stcs(Xqs + i, quant8_f16<false>(cache[i], a));

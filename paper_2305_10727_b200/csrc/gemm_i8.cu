@@ -47,6 +47,7 @@
 
 #include "common.cuh"
 #include "ptx.cuh"
+#include "quant_math.cuh"
 
 namespace gpusq {
 
@@ -155,11 +156,6 @@ __device__ __forceinline__ float2 gelu_pair(float2 y)
     const float2 g = __fmul2_rn(t, make_float2(ex2_approx(r.x), ex2_approx(r.y)));
     // max(y, 0) - g
     return __ffma2_rn(g, make_float2(-1.0f, -1.0f), make_float2(fmaxf(y.x, 0.0f), fmaxf(y.y, 0.0f)));
-}
-
-__device__ __forceinline__ float gelu_one(float y)
-{
-    return gelu_pair(make_float2(y, y)).x;
 }
 
 // FP16 epilogue of one worker warp.  The warp owns 16 tensor-memory lanes (features) and every
@@ -319,7 +315,140 @@ struct EpiF16 {
     }
 };
 
-template <bool kSparse>
+// INT8 epilogue of one worker warp (requantised output).  The warp owns the 32 tensor-memory lanes
+// (features) of its quarter and every fourth 32-token chunk; tcgen05.ld in the 32x32b shape gives each
+// thread one feature and consecutive tokens.  Four tokens of a feature are quantised and packed into a
+// word; two shuffle + byte-permute steps transpose 4 x 4 bytes among four neighbouring lanes, so that
+// each lane holds four neighbouring features of one token and writes them with one 4-byte store into
+// a 128-byte-swizzled [32 tokens][128 features] staging tile that the four quarters' warps share.
+struct EpiI8 {
+    const GemmParams *p;
+    Ctl *ctl;
+    uint8_t *epi_smem;
+    uint32_t tmem_base, tmem_empty0, tmem_empty1;
+    float x_scale, out_scale;
+    int warp, lane, rank, cluster_id, num_clusters, tiles_n, num_tiles, block_t;
+
+    __device__ __forceinline__ void release(int acc)
+    {
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive_cluster(acc ? tmem_empty1 : tmem_empty0);
+    }
+
+    template <bool kGelu>
+    __device__ __forceinline__ void run()
+    {
+        const int quarter = warp & 3;
+        const int sub = (warp - 2) >> 2;                   // 0..3: which chunks, and which staging ring
+        const int g = lane >> 2, l = lane & 3;
+        const uint32_t sel1 = (l & 1) ? 0x3715u : 0x6240u, sel2 = (l & 2) ? 0x3276u : 0x5410u;
+        // this lane's 4 bytes inside a staging row: features 32 q + 4 g .. + 3
+        const int c16 = 2 * quarter + (g >> 2), within = 4 * (g & 3);
+        const uint32_t ring0 = ptx::smem_u32(epi_smem + sub * kEpiBufs * kEpiBufBytes);
+        const uint32_t full0 = ptx::smem_u32(&ctl->stg_full[sub][0]), free0 = ptx::smem_u32(&ctl->stg_free[sub][0]);
+        uint32_t buf_addr = ring0, full_bar = full0, free_bar = free0, buf_idx = 0, free_parity = 1;
+        const int chunks = block_t / kChunkT;
+        const int64_t M = p->M;
+        const int N = p->N;
+        const float *w_scale = p->w_scale, *bias = p->bias;
+        const QuantScale qs = make_quant_scale(out_scale);
+
+        float ws_next, bi_next;
+        auto fetch = [&](int tile) {
+            const int n = (tile % tiles_n) * kPairF + rank * kBlockF + quarter * 32 + lane;
+            const bool in = tile < num_tiles && n < N;
+            ws_next = in ? __ldg(w_scale + n) : 0.0f;
+            bi_next = (in && bias) ? __ldg(bias + n) : 0.0f;
+        };
+        fetch(cluster_id);
+        int local = 0;
+        for (int tile = cluster_id; tile < num_tiles; tile += num_clusters, ++local) {
+            const int tn = tile % tiles_n, tm = tile / tiles_n;
+            const int acc = local & 1;
+            const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
+            const int64_t m0 = (int64_t)tm * block_t;
+            const bool n_valid = tn * kPairF + rank * kBlockF < N;
+            const float sc = __fmul_rn(ws_next, x_scale);
+            const float2 sc2 = make_float2(sc, sc), bi2 = make_float2(bi_next, bi_next);
+            fetch(tile + num_clusters);
+            bool to;
+            if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->tmem_full[acc]), acc_phase, &ctl->abort_flag, to)) {
+                if (to && lane == 0) report_timeout(*p, ctl, tile, 2, 100 + acc);
+                return;
+            }
+            ptx::tc_fence_after();
+            int nchunks = 0;
+            if (n_valid) {
+                const int64_t left = M - m0;
+                nchunks = left >= block_t ? chunks : (int)((left + kChunkT - 1) / kChunkT);
+            }
+            const int c0 = (sub - local) & 3;              // chunk c belongs to the warps with sub == (c + local) % 4
+            if (c0 >= nchunks) {
+                release(acc);
+                continue;
+            }
+            const uint32_t tbase = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * kAccStride);
+            for (int c = c0; c < nchunks; c += 4) {
+                uint32_t va[16], vb[16];
+                ptx::tmem_ld_32x32b_x16(tbase + (uint32_t)(c * kChunkT), va);
+                ptx::tmem_ld_32x32b_x16(tbase + (uint32_t)(c * kChunkT + 16), vb);
+                ptx::tmem_ld_wait_regs(va);
+                ptx::tmem_ld_wait_regs(vb);
+                if (c + 4 >= nchunks) release(acc);        // all this warp reads of the tile is in registers
+                if (!ptx::mbar_wait_bounded(free_bar, free_parity, &ctl->abort_flag, to)) {
+                    if (to && lane == 0) report_timeout(*p, ctl, tile, 2, 200 + (int)buf_idx);
+                    return;
+                }
+#pragma unroll
+                for (int w = 0; w < 8; ++w) {
+                    // tokens 4w .. 4w+3 of the chunk, this thread's feature
+                    const uint32_t a0 = w < 4 ? va[4 * w] : vb[4 * w - 16], a1 = w < 4 ? va[4 * w + 1] : vb[4 * w - 15];
+                    const uint32_t a2 = w < 4 ? va[4 * w + 2] : vb[4 * w - 14], a3 = w < 4 ? va[4 * w + 3] : vb[4 * w - 13];
+                    float2 y01 = __ffma2_rn(make_float2(__int2float_rn((int32_t)a0), __int2float_rn((int32_t)a1)), sc2, bi2);
+                    float2 y23 = __ffma2_rn(make_float2(__int2float_rn((int32_t)a2), __int2float_rn((int32_t)a3)), sc2, bi2);
+                    if (kGelu) {
+                        y01 = gelu_pair(y01);
+                        y23 = gelu_pair(y23);
+                    }
+                    uint32_t differ = 0;
+                    float2 m01 = quant2_sums<true>(y01, qs, differ), m23 = quant2_sums<true>(y23, qs, differ);
+                    if (differ != 0u || qs.always_divide) {
+                        m01 = quant2_exact<true>(y01, qs);
+                        m23 = quant2_exact<true>(y23, qs);
+                    }
+                    const uint32_t word = pack4_low_bytes(m01, m23);          // byte j: token 4w + j
+                    // 4 x 4 byte transpose over lanes 4g .. 4g+3 (features) x tokens 4w .. 4w+3
+                    const uint32_t r1 = __shfl_xor_sync(0xffffffffu, word, 1);
+                    const uint32_t half2tok = __byte_perm(word, r1, sel1);   // two features x two tokens
+                    const uint32_t r2 = __shfl_xor_sync(0xffffffffu, half2tok, 2);
+                    const uint32_t out = __byte_perm(half2tok, r2, sel2);     // features 4g..4g+3 of token 4w + l
+                    const int tok = 4 * w + l;
+                    const uint32_t addr = buf_addr + (uint32_t)(tok * 128 + ((c16 ^ (tok & 7)) << 4) + within);
+                    asm volatile("st.shared.b32 [%0], %1;" ::"r"(addr), "r"(out) : "memory");
+                }
+                ptx::fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(full_bar);
+                if (++buf_idx == (uint32_t)kEpiBufs) {
+                    buf_idx = 0;
+                    free_parity ^= 1u;
+                    buf_addr = ring0;
+                    full_bar = full0;
+                    free_bar = free0;
+                } else {
+                    buf_addr += kEpiBufBytes;
+                    full_bar += 8;
+                    free_bar += 8;
+                }
+            }
+        }
+    }
+};
+
+// kOut = GPUSQ_OUT_F16 / _I8 / _I32: one instantiation per output type, so that each epilogue gets its
+// own register allocation
+template <bool kSparse, int kOut>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kNumThreads, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_e, const __grid_constant__ CUtensorMap map_y,
@@ -371,7 +500,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         ptx::prefetch_tensormap(&map_a);
         ptx::prefetch_tensormap(&map_b);
         if (kSparse) ptx::prefetch_tensormap(&map_e);
-        if (p.out_type == GPUSQ_OUT_F16) ptx::prefetch_tensormap(&map_y);
+        if (kOut != GPUSQ_OUT_I32) ptx::prefetch_tensormap(&map_y);
     }
     if (warp == 1) {
         ptx::tmem_alloc_pair(ptx::smem_u32(&ctl->tmem_base), kTmemCols);
@@ -499,7 +628,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // --------------------------------------------------------- TMA stores
         // One lane per 64-feature half: waits for a staging tile to be filled, stores it, and hands
         // tiles back to the epilogue warps once the stores have read them.
-        if (p.out_type == GPUSQ_OUT_F16 && ptx::elect_one()) {
+        if (kOut == GPUSQ_OUT_F16 && ptx::elect_one()) {
             const int fgroup = warp - kStoreWarp0;         // features [64 fgroup, 64 fgroup + 64) of the CTA's 128
             const int chunks = block_t / kChunkT;
             uint32_t filled0 = 0, filled1 = 0;             // staging tiles stored so far, per chunk parity group
@@ -539,13 +668,52 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             // the staging tiles must stay valid until the bulk stores have read them, and the
             // stores must be complete before the kernel ends
             ptx::tma_store_wait_all<0>();
+        } else if (kOut == GPUSQ_OUT_I8 && ptx::elect_one()) {
+            // INT8 output: staging tiles hold all 128 features of a chunk; rings 0..3 belong to the warps
+            // with that chunk index modulo 4 (rotating per tile); this lane serves rings `odd` and `odd + 2`
+            const int odd = warp - kStoreWarp0;
+            const int chunks = block_t / kChunkT;
+            uint32_t filled_lo = 0, filled_hi = 0;         // staging tiles stored so far from ring odd / odd + 2
+            uint32_t prev1 = 0, prev2 = 0;
+            int local = 0;
+            bool ok = true;
+            for (int tile = cluster_id; ok && tile < num_tiles; tile += num_clusters, ++local) {
+                const int tn = tile % tiles_n, tm = tile / tiles_n;
+                const int64_t m0 = (int64_t)tm * block_t;
+                const int n0 = tn * kPairF + (int)rank * kBlockF;
+                if (n0 >= p.N) continue;
+                const int64_t left = p.M - m0;
+                const int nchunks = left >= block_t ? chunks : (int)((left + kChunkT - 1) / kChunkT);
+                for (int c = 0; c < nchunks; ++c) {
+                    const int ring = (c + local) & 3;
+                    if ((ring & 1) != odd) continue;
+                    const uint32_t count = (ring & 2) ? filled_hi : filled_lo;
+                    const uint32_t b = count % kEpiBufs;
+                    bool to;
+                    if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->stg_full[ring][b]), (count / kEpiBufs) & 1u,
+                                                abort_flag, to)) {
+                        if (to) report_timeout(p, ctl, tile, 3, ring * 8 + (int)b);
+                        ok = false;
+                        break;
+                    }
+                    ptx::tma_store_2d(&map_y, ptx::smem_u32(epi_smem + (ring * kEpiBufs + (int)b) * kEpiBufBytes), n0,
+                                      (int32_t)(m0 + c * kChunkT));
+                    ptx::tma_store_commit();
+                    ptx::tma_store_wait_read<2>();
+                    if (prev2) ptx::mbar_arrive(prev2);
+                    prev2 = prev1;
+                    prev1 = ptx::smem_u32(&ctl->stg_free[ring][b]);
+                    if (ring & 2) ++filled_hi; else ++filled_lo;
+                }
+            }
+            ptx::tma_store_wait_all<0>();
         }
     } else {
         // ------------------------------------------------------------ epilogue
         const int quarter = warp & 3;                      // tensor-memory lanes [32q, 32q+32) are this warp's to read
         const int par = (warp - 2) >> 3;                   // FP16 path: which chunks, every other one
-        const float x_scale = (p.out_type == GPUSQ_OUT_I32) ? 1.0f : __ldg(p.x_scale);
-        const float out_scale = (p.out_type == GPUSQ_OUT_I8) ? __ldg(p.out_scale) : 1.0f;
+        const float x_scale = (kOut == GPUSQ_OUT_I32) ? 1.0f : __ldg(p.x_scale);
+        const float out_scale = (kOut == GPUSQ_OUT_I8) ? __ldg(p.out_scale) : 1.0f;
         // the accumulators of both CTAs are released on CTA 0's barrier, where the MMA issuer waits
         const uint32_t tmem_empty0 = ptx::map_to_cta(ptx::smem_u32(&ctl->tmem_empty[0]), 0);
         const uint32_t tmem_empty1 = ptx::map_to_cta(ptx::smem_u32(&ctl->tmem_empty[1]), 0);
@@ -553,7 +721,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const uint32_t stage0 = ptx::smem_u32(epi_smem + group * kEpiBufs * kEpiBufBytes);
         int local = 0;
 
-        if (p.out_type == GPUSQ_OUT_F16) {
+        if (kOut == GPUSQ_OUT_F16) {
             EpiF16 e;
             e.p = &p;
             e.ctl = ctl;
@@ -576,7 +744,31 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 e.template run<true>();
             else
                 e.template run<false>();
+        } else if (kOut == GPUSQ_OUT_I8) {
+            EpiI8 e;
+            e.p = &p;
+            e.ctl = ctl;
+            e.epi_smem = epi_smem;
+            e.tmem_base = tmem_base;
+            e.tmem_empty0 = tmem_empty0;
+            e.tmem_empty1 = tmem_empty1;
+            e.x_scale = x_scale;
+            e.out_scale = out_scale;
+            e.warp = warp;
+            e.lane = lane;
+            e.rank = (int)rank;
+            e.cluster_id = cluster_id;
+            e.num_clusters = num_clusters;
+            e.tiles_n = tiles_n;
+            e.num_tiles = num_tiles;
+            e.block_t = block_t;
+            if (p.act == GPUSQ_ACT_GELU)
+                e.template run<true>();
+            else
+                e.template run<false>();
         } else {
+            // raw INT32 accumulators (for bit-exact comparison): plain coalesced stores; the four warps
+            // of a quarter take every fourth 16-token chunk
             for (int tile = cluster_id; tile < num_tiles; tile += num_clusters, ++local) {
                 const int tn = tile % tiles_n, tm = tile / tiles_n;
                 const int acc = local & 1;
@@ -584,13 +776,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 const int64_t m0 = (int64_t)tm * block_t;
                 const int n0 = tn * kPairF + (int)rank * kBlockF;
                 const bool n_valid = n0 < p.N;
-                const uint32_t tmem_empty = acc ? tmem_empty1 : tmem_empty0;
                 const int n = n0 + quarter * 32 + lane;                // this thread's output feature
-                float sc = 1.0f, bi = 0.0f;
-                if (p.out_type != GPUSQ_OUT_I32 && n_valid) {
-                    sc = __fmul_rn(__ldg(p.w_scale + n), x_scale);
-                    bi = p.bias ? __ldg(p.bias + n) : 0.0f;
-                }
                 bool to;
                 if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->tmem_full[acc]), acc_phase, abort_flag, to)) {
                     if (to && lane == 0) report_timeout(p, ctl, tile, 2, 100 + acc);
@@ -598,7 +784,6 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 }
                 ptx::tc_fence_after();
                 const uint32_t tbase = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * kAccStride);
-                // the four warps of a quarter take every fourth 16-token chunk
                 for (int c = (warp - 2) >> 2; c < block_t / 16 && n_valid; c += kEpiWarps / 4) {
                     if (m0 + c * 16 >= p.M) break;
                     uint32_t r[16];
@@ -607,23 +792,12 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
                         const int64_t m = m0 + c * 16 + j;
-                        if (m < p.M) {
-                            const int32_t a = (int32_t)r[j];
-                            if (p.out_type == GPUSQ_OUT_I32) {
-                                reinterpret_cast<int32_t *>(p.Y)[m * p.N + n] = a;
-                            } else {
-                                float y = __fmaf_rn(__int2float_rn(a), sc, bi);
-                                if (p.act == GPUSQ_ACT_GELU) y = gelu_one(y);
-                                int q = __float2int_rn(__fdiv_rn(y, out_scale));
-                                q = max(-127, min(127, q));
-                                reinterpret_cast<int8_t *>(p.Y)[m * p.N + n] = (int8_t)q;
-                            }
-                        }
+                        if (m < p.M) reinterpret_cast<int32_t *>(p.Y)[m * p.N + n] = (int32_t)r[j];
                     }
                 }
                 ptx::tc_fence_before();
                 __syncwarp();
-                if (lane == 0) ptx::mbar_arrive_cluster(tmem_empty);
+                if (lane == 0) ptx::mbar_arrive_cluster(acc ? tmem_empty1 : tmem_empty0);
             }
         }
     }
@@ -723,7 +897,7 @@ static int max_clusters(int sms)
         cfg.blockDim = dim3(kNumThreads, 1, 1);
         cfg.dynamicSmemBytes = Cfg<kSparse>::kSmemBytes;
         int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, gemm_i8_kernel<kSparse>, &cfg) != cudaSuccess || n <= 0) {
+        if (cudaOccupancyMaxActiveClusters(&n, gemm_i8_kernel<kSparse, GPUSQ_OUT_F16>, &cfg) != cudaSuccess || n <= 0) {
             (void)cudaGetLastError();
             n = sms / 2;
         }
@@ -749,11 +923,13 @@ static int launch_gemm(const int8_t *Xq, const void *Wsrc, const float *w_scale,
     static std::once_flag attr_once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(attr_once, [] {
-        attr_err = cudaFuncSetAttribute(gemm_i8_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        Cfg<true>::kSmemBytes);
-        if (attr_err == cudaSuccess)
-            attr_err = cudaFuncSetAttribute(gemm_i8_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            Cfg<false>::kSmemBytes);
+        const void *kernels[6] = {
+            (const void *)gemm_i8_kernel<true, GPUSQ_OUT_F16>,  (const void *)gemm_i8_kernel<true, GPUSQ_OUT_I8>,
+            (const void *)gemm_i8_kernel<true, GPUSQ_OUT_I32>,  (const void *)gemm_i8_kernel<false, GPUSQ_OUT_F16>,
+            (const void *)gemm_i8_kernel<false, GPUSQ_OUT_I8>,  (const void *)gemm_i8_kernel<false, GPUSQ_OUT_I32>};
+        for (int k = 0; k < 6 && attr_err == cudaSuccess; ++k)
+            attr_err = cudaFuncSetAttribute(kernels[k], cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            k < 3 ? Cfg<true>::kSmemBytes : Cfg<false>::kSmemBytes);
     });
     if (attr_err != cudaSuccess) return GPUSQ_ERR_CUDA;
 
@@ -781,6 +957,9 @@ static int launch_gemm(const int8_t *Xq, const void *Wsrc, const float *w_scale,
     }
     CUtensorMap map_y = map_b;      // placeholder unless the output is FP16
     if (out_type == GPUSQ_OUT_F16) ok = ok && make_map_y_f16(&map_y, Y, (uint64_t)M, (uint64_t)N);
+    // INT8 output: box = 128 features x 32 tokens, 128-byte swizzle (the INT8 staging-tile layout)
+    if (out_type == GPUSQ_OUT_I8)
+        ok = ok && make_map_u8(&map_y, Y, (uint64_t)M, (uint64_t)N, 128, (uint32_t)kChunkT, CU_TENSOR_MAP_SWIZZLE_128B);
     if (!ok) return GPUSQ_ERR_CUDA;
 
     GemmParams p;
@@ -809,7 +988,14 @@ static int launch_gemm(const int8_t *Xq, const void *Wsrc, const float *w_scale,
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, gemm_i8_kernel<kSparse>, map_a, map_b, map_e, map_y, p) != cudaSuccess) {
+    cudaError_t err;
+    if (out_type == GPUSQ_OUT_F16)
+        err = cudaLaunchKernelEx(&cfg, gemm_i8_kernel<kSparse, GPUSQ_OUT_F16>, map_a, map_b, map_e, map_y, p);
+    else if (out_type == GPUSQ_OUT_I8)
+        err = cudaLaunchKernelEx(&cfg, gemm_i8_kernel<kSparse, GPUSQ_OUT_I8>, map_a, map_b, map_e, map_y, p);
+    else
+        err = cudaLaunchKernelEx(&cfg, gemm_i8_kernel<kSparse, GPUSQ_OUT_I32>, map_a, map_b, map_e, map_y, p);
+    if (err != cudaSuccess) {
         (void)cudaGetLastError();
         return GPUSQ_ERR_CUDA;
     }

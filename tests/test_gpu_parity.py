@@ -209,17 +209,29 @@ def test_epilogue_gelu_wide_range(B):
     assert f16_ulp_distance(Y, Y_o).max() <= F16_ULP_TOL
 
 
+@pytest.mark.parametrize("M,N,K,block_t", [(514, 256, 1280, 0), (197, 128, 192, 0), (1000, 384, 256, 96),
+                                           (33, 128, 64, 32), (1576, 768, 192, 224)])
 @pytest.mark.parametrize("act", [0, 1])
-def test_epilogue_int8_requantised(B, act):
-    M, N, K = 514, 256, 1280
+def test_epilogue_int8_requantised(B, act, M, N, K, block_t):
     d, prep, Xq, xs = _prep(5, M, N, K)
     acc_o = oracle.spgemm_acc(Xq, prep["vals"], prep["meta"])
     yf = oracle.epilogue(acc_o, prep["w_scale"], xs, d["bias"], act=act, out_type=0).astype(np.float32)
     out_scale = np.float32(np.abs(yf).max() / 127.0)
     Q_o = oracle.epilogue(acc_o, prep["w_scale"], xs, d["bias"], act=act, out_type=1, out_scale=out_scale)
-    Q = B.spgemm_i8(cu(Xq), B.pack24(cu(prep["vals"]), cu(prep["meta"])), N, w_scale=cu(prep["w_scale"]),
-                    x_scale=cu(np.array([xs], np.float32)), bias=cu(d["bias"]), act=act, out_type=B.OUT_I8,
-                    out_scale=cu(np.array([out_scale], np.float32))).cpu().numpy()
+    status = torch.zeros(4, dtype=torch.int32, device="cuda")
+    B.set_block_tokens(block_t)
+    try:
+        Q = B.spgemm_i8(cu(Xq), B.pack24(cu(prep["vals"]), cu(prep["meta"])), N, w_scale=cu(prep["w_scale"]),
+                        x_scale=cu(np.array([xs], np.float32)), bias=cu(d["bias"]), act=act, out_type=B.OUT_I8,
+                        out_scale=cu(np.array([out_scale], np.float32)), status_buf=status).cpu().numpy()
+        Qd = B.gemm_i8_dense(cu(Xq), cu(prep["Wq"]), w_scale=cu(prep["w_scale"]),
+                             x_scale=cu(np.array([xs], np.float32)), bias=cu(d["bias"]), act=act,
+                             out_type=B.OUT_I8, out_scale=cu(np.array([out_scale], np.float32)),
+                             status_buf=status).cpu().numpy()
+    finally:
+        B.set_block_tokens(0)
+    assert status.cpu().tolist() == [0, 0, 0, 0]
+    assert np.array_equal(Q, Qd)                         # the dense variant runs the same epilogue
     diff = np.abs(Q.astype(np.int32) - Q_o.astype(np.int32))
     if act == 0:
         assert diff.max() == 0                           # integer decision taken in the same FP32 sequence
