@@ -240,6 +240,37 @@ def test_epilogue_int8_requantised(B, act, M, N, K, block_t):
         assert diff.max() <= 1 and (diff != 0).mean() < 1e-3
 
 
+def test_int8_chained_mlp(B):
+    # fc1 (GELU) writes requantised INT8 codes that fc2 reads with the same scale: the deployed model's
+    # quantise / de-quantise chain (Sec. 2.2).  fc1's codes may differ from the oracle's by one code at
+    # rounding ties of the GELU (< 0.1 % of them); fc2's output may then differ by at most that many
+    # code steps times the largest de-quantised weight, per row, plus the FP16 rounding.
+    M, H, F = 333, 128, 512
+    d1 = inputs.random_layer(21, M, F, H)
+    d2 = inputs.random_layer(22, M, H, F)
+    p1, p2 = oracle.prepare_weight(d1["W"]), oracle.prepare_weight(d2["W"])
+    r1 = oracle.layer_forward(d1["X"], p1, d1["bias"], act=1)
+    y_scale = np.float32(np.abs(r1["Y"].astype(np.float32)).max() / 127.0)
+    q1_o = oracle.epilogue(r1["acc"], p1["w_scale"], r1["x_scale"], d1["bias"], act=1, out_type=1, out_scale=y_scale)
+    acc2_o = oracle.spgemm_acc(q1_o, p2["vals"], p2["meta"])
+    y2_o = oracle.epilogue(acc2_o, p2["w_scale"], y_scale, d2["bias"], act=0, out_type=0).astype(np.float32)
+
+    Xq, xs = B.quant_act(cu(d1["X"]))
+    ys = cu(np.array([y_scale], np.float32))
+    q1 = B.spgemm_i8(Xq, B.pack24(cu(p1["vals"]), cu(p1["meta"])), F, cu(p1["w_scale"]), xs, cu(d1["bias"]),
+                     act=B.ACT_GELU, out_type=B.OUT_I8, out_scale=ys)
+    y2 = B.spgemm_i8(q1, B.pack24(cu(p2["vals"]), cu(p2["meta"])), H, cu(p2["w_scale"]), ys, cu(d2["bias"]),
+                     act=B.ACT_NONE, out_type=B.OUT_F16).cpu().numpy().astype(np.float32)
+    steps = np.abs(q1.cpu().numpy().astype(np.int32) - q1_o.astype(np.int32))
+    assert steps.max() <= 1 and (steps != 0).mean() < 1e-3
+    w_max = float((np.abs(p2["Wq"]).max(axis=1) * p2["w_scale"]).max())
+    bound = steps.sum(axis=1, keepdims=True) * w_max * float(y_scale) + np.abs(y2_o) * 2.0 ** -10 + 2.0 ** -24
+    assert (np.abs(y2 - y2_o) <= bound).all()
+    # rows whose codes all agree are reproduced to the bit
+    same = steps.sum(axis=1) == 0
+    assert same.any() and np.array_equal(y2[same], y2_o[same])
+
+
 def test_whole_path_on_device_matches_oracle(B):
     # every step of the path on the GPU, chained, against the oracle chained the same way
     cfg = inputs.CONFIGS["deit_tiny_fc1"]
