@@ -345,6 +345,8 @@ struct EpiI8 {
         const uint32_t sel1 = (l & 1) ? 0x3715u : 0x6240u, sel2 = (l & 2) ? 0x3276u : 0x5410u;
         // this lane's 4 bytes inside a staging row: features 32 q + 4 g .. + 3
         const int c16 = 2 * quarter + (g >> 2), within = 4 * (g & 3);
+        const uint32_t row_off0 = (uint32_t)(l * 128 + ((c16 ^ l) << 4) + within);
+        const uint32_t row_off1 = (uint32_t)(l * 128 + ((c16 ^ (4 + l)) << 4) + within);
         const uint32_t ring0 = ptx::smem_u32(epi_smem + sub * kEpiBufs * kEpiBufBytes);
         const uint32_t full0 = ptx::smem_u32(&ctl->stg_full[sub][0]), free0 = ptx::smem_u32(&ctl->stg_free[sub][0]);
         uint32_t buf_addr = ring0, full_bar = full0, free_bar = free0, buf_idx = 0, free_parity = 1;
@@ -411,9 +413,12 @@ struct EpiI8 {
                         y01 = gelu_pair(y01);
                         y23 = gelu_pair(y23);
                     }
+                    // values beyond +-127 out_scale saturate: rare, so they are only detected here (one
+                    // compare per four values) and handled, clamp included, by the exact branch
+                    const bool beyond = fmaxf(fmaxf(fabsf(y01.x), fabsf(y01.y)), fmaxf(fabsf(y23.x), fabsf(y23.y))) > qs.x_max;
                     uint32_t differ = 0;
-                    float2 m01 = quant2_sums<true>(y01, qs, differ), m23 = quant2_sums<true>(y23, qs, differ);
-                    if (differ != 0u || qs.always_divide) {
+                    float2 m01 = quant2_sums<false>(y01, qs, differ), m23 = quant2_sums<false>(y23, qs, differ);
+                    if (differ != 0u || beyond || qs.always_divide) {
                         m01 = quant2_exact<true>(y01, qs);
                         m23 = quant2_exact<true>(y23, qs);
                     }
@@ -423,8 +428,8 @@ struct EpiI8 {
                     const uint32_t half2tok = __byte_perm(word, r1, sel1);   // two features x two tokens
                     const uint32_t r2 = __shfl_xor_sync(0xffffffffu, half2tok, 2);
                     const uint32_t out = __byte_perm(half2tok, r2, sel2);     // features 4g..4g+3 of token 4w + l
-                    const int tok = 4 * w + l;
-                    const uint32_t addr = buf_addr + (uint32_t)(tok * 128 + ((c16 ^ (tok & 7)) << 4) + within);
+                    // row 4w + l of the tile; (4w + l) & 7 = l or 4 + l, so two offsets serve all eight words
+                    const uint32_t addr = buf_addr + ((w & 1) ? row_off1 : row_off0) + (uint32_t)(w * 512);
                     asm volatile("st.shared.b32 [%0], %1;" ::"r"(addr), "r"(out) : "memory");
                 }
                 ptx::fence_proxy_async_smem();

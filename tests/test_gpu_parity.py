@@ -212,12 +212,14 @@ def test_epilogue_gelu_wide_range(B):
 @pytest.mark.parametrize("M,N,K,block_t", [(514, 256, 1280, 0), (197, 128, 192, 0), (1000, 384, 256, 96),
                                            (33, 128, 64, 32), (1576, 768, 192, 224)])
 @pytest.mark.parametrize("act", [0, 1])
-def test_epilogue_int8_requantised(B, act, M, N, K, block_t):
+@pytest.mark.parametrize("shrink", [1.0, 0.3])           # 0.3: a third of the range saturates at +-127
+def test_epilogue_int8_requantised(B, act, M, N, K, block_t, shrink):
     d, prep, Xq, xs = _prep(5, M, N, K)
     acc_o = oracle.spgemm_acc(Xq, prep["vals"], prep["meta"])
     yf = oracle.epilogue(acc_o, prep["w_scale"], xs, d["bias"], act=act, out_type=0).astype(np.float32)
-    out_scale = np.float32(np.abs(yf).max() / 127.0)
+    out_scale = np.float32(shrink * np.abs(yf).max() / 127.0)
     Q_o = oracle.epilogue(acc_o, prep["w_scale"], xs, d["bias"], act=act, out_type=1, out_scale=out_scale)
+    assert shrink == 1.0 or (np.abs(Q_o) == 127).mean() > 1e-3
     status = torch.zeros(4, dtype=torch.int32, device="cuda")
     B.set_block_tokens(block_t)
     try:
