@@ -81,16 +81,38 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 // looks at the flag and the clock only every 32 tries.
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s
 constexpr uint32_t kRetrySleepNs = 100;
+// Up to 32 tries with a short sleep after each failed one, as one tight loop (try, branch, sleep,
+// count): waiting warps should cost the working ones as few issue slots as possible.
+__device__ __forceinline__ bool mbar_try_wait_32(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred P, Q;\n"
+        ".reg .u32 n;\n"
+        "mov.u32 n, 32;\n"
+        "TRY_AGAIN:\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 P, [%1], %2;\n"
+        "@P bra DONE;\n"
+        "nanosleep.u32 %3;\n"
+        "sub.u32 n, n, 1;\n"
+        "setp.ne.u32 Q, n, 0;\n"
+        "@Q bra TRY_AGAIN;\n"
+        "DONE:\n"
+        "selp.u32 %0, 1, 0, P;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(kRetrySleepNs)
+        : "memory");
+    return ok != 0;
+}
+
 // returns 0 = phase complete, 1 = abort flag seen, 2 = time limit reached
 __device__ __noinline__ int mbar_wait_slow(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag)
 {
     const uint64_t t0 = globaltimer_ns();
     for (;;) {
-#pragma unroll 1
-        for (int it = 0; it < 32; ++it) {
-            if (mbar_try_wait(bar, parity)) return 0;
-            __nanosleep(kRetrySleepNs);          // leave the issue slots to the warps that have work
-        }
+        if (mbar_try_wait_32(bar, parity)) return 0;
         if (*abort_flag) return 1;
         if (globaltimer_ns() - t0 > kWaitLimitNs) return 2;
     }
