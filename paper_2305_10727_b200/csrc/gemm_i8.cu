@@ -870,17 +870,20 @@ static bool make_map_y_f16(CUtensorMap *map, void *base, uint64_t M, uint64_t N)
 
 static int g_block_t_override = 0;
 
-// Tokens per tile: a multiple of 32 up to 224 chosen so that the last wave of
-// tiles over the SM pairs is as full as possible (per-tile cost ~ block_t + fixed part).
-static int choose_block_t(int64_t M, int tiles_n, int clusters)
+// Tokens per tile: a multiple of 32 up to 224 that minimises waves x time per tile.  Per tile and CTA
+// the shared memory moves, per 128-wide k block, 128 bytes per token (activations written and read)
+// plus a fixed ~20 KB for the weight block (as much as 160 tokens), and the epilogue's staging costs
+// as much as four k blocks per token: time per tile ~ (kb + 4) * block_t + 160 * kb.
+static int choose_block_t(int64_t M, int tiles_n, int clusters, int K)
 {
     if (g_block_t_override) return g_block_t_override;
+    const double kb = (double)ceil_div(K, kBlockK);
     int best = kMaxBlockT;
     double best_cost = 1e300;
     for (int bt = kMaxBlockT; bt >= 32; bt -= 32) {
         const int64_t tiles = (int64_t)tiles_n * ceil_div(M, bt);
         const int64_t waves = ceil_div(tiles, clusters);
-        const double cost = (double)waves * (bt + 48);
+        const double cost = (double)waves * ((kb + 4.0) * bt + 160.0 * kb);
         if (cost < best_cost * 0.999) {
             best_cost = cost;
             best = bt;
@@ -944,7 +947,7 @@ static int launch_gemm(const int8_t *Xq, const void *Wsrc, const float *w_scale,
     const int clusters = max_clusters<kSparse>(sms);
     if (clusters <= 0) return GPUSQ_ERR_CUDA;
     const int tiles_n = (N + kPairF - 1) / kPairF;
-    const int block_t = choose_block_t(M, tiles_n, clusters);
+    const int block_t = choose_block_t(M, tiles_n, clusters, K);
     const int Kp = round_up(K, 128), Np = round_up(N, kPairF);
 
     CUtensorMap map_a, map_b;
