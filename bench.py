@@ -403,7 +403,8 @@ def run_gpusq(args, cfg):
         }
     roofline = {
         "bound": "tensor", "kernel": "gemm_i8_kernel<sparse>", "achieved": round(achieved, 1),
-        "peak": round(peak, 1), "unit": "TFLOP/s", "frac": round(achieved / peak, 4), "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH,
+        "peak": round(peak, 1), "unit": "TFLOP/s", "frac": round(achieved / peak, 4),
+        "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH if args.config == "deit_base_b64" else None,
         "peak_source": "%s BF16 sustained x %.0f (nominal INT8-sparse : BF16 ratio)" % (peaks["_source"], sparse_ratio),
         "frac_of_nominal_9000": round(achieved / NOMINAL_SPARSE_INT8_TOPS, 4),
         "frac_of_burst_peak": round(achieved / (peaks["bf16_tflops"] * sparse_ratio), 4),

@@ -180,7 +180,10 @@ int gpusq_quant_act_static(const void *X, int8_t *Xq, float *x_scale, int scale_
  *     a kernel whose bounded wait expires writes {GPUSQ_ERR_TIMEOUT, tile,
  *     role, stage} there and stops issuing work (the output is then
  *     undefined).  The host call itself never waits for the device.
- * Requires M > 0, N % 128 == 0, K % 16 == 0, Xq / Wpacked / Y 16-byte aligned.
+ * Requires M > 0, K % 16 == 0, Xq / Wpacked / Y 16-byte aligned, and a row of
+ * Y that is a multiple of 16 bytes: N % 8 == 0 for GPUSQ_OUT_F16, N % 16 == 0
+ * for GPUSQ_OUT_I8 (any N for GPUSQ_OUT_I32).  N need not be a multiple of
+ * the 128-feature tile (DeiT-Tiny's 192 and 576, Swin-Tiny's 96 and 288).
  */
 int gpusq_spgemm_i8(const int8_t *Xq, const void *Wpacked, const float *w_scale,
                     const float *x_scale, const float *bias, int act, int out_type,

@@ -264,8 +264,9 @@ struct EpiF16 {
             const bool in = tile < num_tiles && n0 < N;
 #pragma unroll
             for (int j = 0; j < 2; ++j) {
-                ws_next[j] = in ? __ldg(w_scale + n0 + nofs + 8 * j) : 0.0f;
-                bi_next[j] = (in && bias) ? __ldg(bias + n0 + nofs + 8 * j) : 0.0f;
+                const int n = n0 + nofs + 8 * j;           // N need not fill the last 128-feature block
+                ws_next[j] = (in && n < N) ? __ldg(w_scale + n) : 0.0f;
+                bi_next[j] = (in && n < N && bias) ? __ldg(bias + n) : 0.0f;
             }
         };
         fetch(cluster_id);
@@ -799,7 +800,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
                         const int64_t m = m0 + c * 16 + j;
-                        if (m < p.M) reinterpret_cast<int32_t *>(p.Y)[m * p.N + n] = (int32_t)r[j];
+                        if (m < p.M && n < p.N) reinterpret_cast<int32_t *>(p.Y)[m * p.N + n] = (int32_t)r[j];
                     }
                 }
                 ptx::tc_fence_before();
@@ -926,7 +927,9 @@ static int launch_gemm(const int8_t *Xq, const void *Wsrc, const float *w_scale,
     if (out_type < 0 || out_type > 2 || act < 0 || act > 1) return GPUSQ_ERR_ARG;
     if (out_type != GPUSQ_OUT_I32 && (!w_scale || !x_scale)) return GPUSQ_ERR_NULL;
     if (out_type == GPUSQ_OUT_I8 && !out_scale) return GPUSQ_ERR_NULL;
-    if (M <= 0 || N <= 0 || K <= 0 || N % kBlockF || K % 16 || M > 0x7FFFFFFF) return GPUSQ_ERR_SHAPE;
+    if (M <= 0 || N <= 0 || K <= 0 || K % 16 || M > 0x7FFFFFFF) return GPUSQ_ERR_SHAPE;
+    // rows of Y are written by bulk tensor stores, whose row pitch is a multiple of 16 bytes
+    if ((out_type == GPUSQ_OUT_F16 && N % 8) || (out_type == GPUSQ_OUT_I8 && N % 16)) return GPUSQ_ERR_SHAPE;
     if (!aligned(Xq, 16) || !aligned(Wsrc, 16) || !aligned(Y, 16)) return GPUSQ_ERR_ALIGN;
     if (int st = check_arch()) return st;
 

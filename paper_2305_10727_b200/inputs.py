@@ -6,8 +6,8 @@ library and the CPU oracle are given, and names the layer shapes.
 
 Shapes follow the models the paper compresses (DeiT / Swin; Sec. 4) and the
 larger ViT-L/H used for scaling: 197 = 14*14+1 tokens per 224x224 image with
-16x16 patches, 196 tokens per image in 7x7 windows for Swin, 257 = 16*16+1
-for ViT-H/14.  Distributions: trained ViT weights are close to a zero-mean
+16x16 patches, 196 tokens per image in 7x7 windows for Swin stage 3 and
+3136 = 56*56 in stage 1 (4x4 patches), 257 = 16*16+1 for ViT-H/14.  Distributions: trained ViT weights are close to a zero-mean
 normal with sigma ~0.02 (the usual truncated-normal initialisation keeps that
 scale), biases are small, LayerNorm outputs are roughly unit normal; the
 heavy-tailed case (Student-t, 4 degrees of freedom, scaled to unit variance)
@@ -61,6 +61,10 @@ CONFIGS: Dict[str, Config] = {
     "vit_huge_b64": Config(4, "ViT-Huge/14 block, batch 64", 64 * 257, _block(1280, 5120), int8_out=True),
     "vit_huge_b256": Config(4, "ViT-Huge/14 block, batch 256", 256 * 257, _block(1280, 5120),
                             int8_out=True),
+    # the paper's smallest models: output widths that are not multiples of the 128-feature tile
+    "deit_tiny_b64": Config(5, "DeiT-Tiny block, batch 64", 64 * 197, _block(192, 768), int8_out=True),
+    "swin_tiny_s1_b32": Config(6, "Swin-Tiny stage 1 block, batch 32", 32 * 3136, _block(96, 384),
+                               x_dist="student_t4", int8_out=True),
 }
 
 _TENSOR_ID = {"W": 0, "bias": 1, "X": 2}

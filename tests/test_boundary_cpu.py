@@ -76,7 +76,9 @@ def test_argument_errors_are_reported_before_any_cuda_call(lib):
         bad = list(ok); bad[0] = None
         assert fn(*bad) == NULL
         bad = list(ok); bad[10] = 100
-        assert fn(*bad) == SHAPE                  # N % 128
+        assert fn(*bad) == SHAPE                  # FP16 rows of Y: N % 8
+        bad = list(ok); bad[10] = 104; bad[6] = 1; bad[7] = p(a16)
+        assert fn(*bad) == SHAPE                  # INT8 rows of Y: N % 16
         bad = list(ok); bad[11] = 40
         assert fn(*bad) == SHAPE                  # K % 16
         bad = list(ok); bad[9] = 0

@@ -139,6 +139,8 @@ def _prep(seed, M, N, K, dist="normal"):
 GEMM_SHAPES = [
     (1, 128, 16), (16, 128, 64), (197, 256, 192), (257, 384, 128), (300, 128, 1280),
     (1576, 768, 192), (1000, 512, 2048),
+    # output widths that do not fill the last 128-feature tile (DeiT-Tiny 192 / 576, Swin-Tiny 96 / 288), K < 128
+    (394, 96, 48), (197, 192, 192), (500, 288, 96), (333, 576, 192), (70, 8, 16), (129, 200, 64), (65, 5, 32),
 ]
 
 
@@ -176,7 +178,8 @@ def test_spgemm_extreme_codes_do_not_overflow(B):
     assert np.array_equal(Y.cpu().numpy(), acc_o)
 
 
-@pytest.mark.parametrize("M,N,K", [(197, 256, 192), (1576, 768, 192), (333, 128, 1024)])
+@pytest.mark.parametrize("M,N,K", [(197, 256, 192), (1576, 768, 192), (333, 128, 1024), (394, 96, 48),
+                                   (591, 576, 192), (100, 200, 64), (77, 8, 16)])
 @pytest.mark.parametrize("act", [0, 1])
 @pytest.mark.parametrize("use_bias", [True, False])
 def test_epilogue_f16(B, M, N, K, act, use_bias):
@@ -210,7 +213,8 @@ def test_epilogue_gelu_wide_range(B):
 
 
 @pytest.mark.parametrize("M,N,K,block_t", [(514, 256, 1280, 0), (197, 128, 192, 0), (1000, 384, 256, 96),
-                                           (33, 128, 64, 32), (1576, 768, 192, 224)])
+                                           (33, 128, 64, 32), (1576, 768, 192, 224), (394, 96, 48, 0),
+                                           (500, 288, 96, 64), (333, 576, 192, 0), (70, 16, 16, 0)])
 @pytest.mark.parametrize("act", [0, 1])
 @pytest.mark.parametrize("shrink", [1.0, 0.3])           # 0.3: a third of the range saturates at +-127
 def test_epilogue_int8_requantised(B, act, M, N, K, block_t, shrink):
