@@ -20,4 +20,8 @@ from .oracle import (  # noqa: F401
     sqnr_db,
     layer_forward,
     prepare_weight,
+    patch_rows,
+    patch_conv_acc,
+    patch_embed_weight,
+    patch_embed_forward,
 )

@@ -205,6 +205,46 @@ int64_t o_spgemm_acc_rows(const int8_t *Xq, const int8_t *vals, const uint8_t *m
     return overflow;
 }
 
+void o_patch_rows(const int8_t *imgq, int8_t *X, int B, int C, int H, int W, int P, int Kp)
+{
+    const int Ty = H / P, Tx = W / P;
+    for (int b = 0; b < B; ++b)
+        for (int ty = 0; ty < Ty; ++ty)
+            for (int tx = 0; tx < Tx; ++tx) {
+                int8_t *row = X + (((int64_t)b * Ty + ty) * Tx + tx) * Kp;
+                for (int k = 0; k < Kp; ++k) row[k] = 0;
+                for (int c = 0; c < C; ++c)
+                    for (int py = 0; py < P; ++py)
+                        for (int px = 0; px < P; ++px)
+                            row[(c * P + py) * P + px] =
+                                imgq[(((int64_t)b * C + c) * H + ty * P + py) * W + tx * P + px];
+            }
+}
+
+int64_t o_patch_conv_acc(const int8_t *imgq, const int8_t *Wq, int32_t *acc, int B, int C,
+                         int H, int W, int P, int D)
+{
+    const int Ty = H / P, Tx = W / P;
+    int64_t macs = 0;
+    for (int b = 0; b < B; ++b)
+        for (int d = 0; d < D; ++d)
+            for (int ty = 0; ty < Ty; ++ty)
+                for (int tx = 0; tx < Tx; ++tx) {
+                    int64_t sum = 0;
+                    for (int c = 0; c < C; ++c)
+                        for (int py = 0; py < P; ++py)
+                            for (int px = 0; px < P; ++px) {
+                                const int64_t w = Wq[(((int64_t)d * C + c) * P + py) * P + px];
+                                const int64_t x =
+                                    imgq[(((int64_t)b * C + c) * H + ty * P + py) * W + tx * P + px];
+                                sum += w * x;
+                                ++macs;
+                            }
+                    acc[(((int64_t)b * Ty + ty) * Tx + tx) * D + d] = (int32_t)sum;
+                }
+    return macs;
+}
+
 void o_epilogue(const int32_t *acc, const float *w_scale, float x_scale,
                 const float *bias, int act, int out_type, float out_scale,
                 void *Y, int64_t count, int N)

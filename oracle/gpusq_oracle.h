@@ -77,6 +77,28 @@ int64_t o_spgemm_acc_rows(const int8_t *Xq, const int8_t *vals, const uint8_t *m
                           const int64_t *rows, int64_t n_rows, int32_t *acc_rows,
                           int N, int K);
 
+/* Sec. 3.3 (patch embedding): an image batch [B, C, H, W] is cut into
+ * non-overlapping P x P patches and the embedding is a convolution with C
+ * input channels, D output channels, kernel size = stride = P, executed as a
+ * GEMM whose reduction axis C*P*P is the axis the 2:4 pattern runs along.
+ * Readings (paper silent): the image is quantised like any activation tensor
+ * (o_quant_act on its B*C*H*W elements, one scale); a token is one patch,
+ * tokens ordered (b, ty, tx) row-major as in the usual flatten of the
+ * convolution output; reduction index k = (c*P + py)*P + px, the row-major
+ * flattening of a convolution weight [D, C, P, P].  H % P == 0, W % P == 0.
+ *
+ * o_patch_rows: the GEMM's activation matrix, X[t, k] = imgq[b, c, ty*P+py,
+ * tx*P+px], columns C*P*P .. Kp-1 zero (Kp >= C*P*P pads the reduction axis
+ * to what the GEMM accepts; the weight is padded with zero columns alike). */
+void o_patch_rows(const int8_t *imgq, int8_t *X, int B, int C, int H, int W, int P, int Kp);
+
+/* The convolution written as its definition on the INT8 codes:
+ * acc[(b, ty, tx), d] = sum_{c, py, px} Wq[d, c, py, px] * imgq[b, c, ty*P+py, tx*P+px]
+ * (64-bit sums, stored as INT32).  Returns the number of multiply-adds done:
+ * B*C*H*W*D, half the FLOP count Sec. 3.3 states. */
+int64_t o_patch_conv_acc(const int8_t *imgq, const int8_t *Wq, int32_t *acc, int B, int C,
+                         int H, int W, int P, int D);
+
 /* Sec. 2.2 (de-quantise node; GELU is the activation the paper names).
  * Reading, in binary32 in this order: t = (float)acc (round-to-nearest-even);
  * s = w_scale[n] * x_scale; y = fma(t, s, bias ? bias[n] : 0);

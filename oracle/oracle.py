@@ -53,6 +53,10 @@ def _load():
             lib.o_spgemm_acc.restype = i64
             lib.o_spgemm_acc_rows.argtypes = [vp, vp, vp, vp, i64, vp, i32, i32]
             lib.o_spgemm_acc_rows.restype = i64
+            lib.o_patch_rows.argtypes = [vp, vp, i32, i32, i32, i32, i32, i32]
+            lib.o_patch_rows.restype = None
+            lib.o_patch_conv_acc.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32]
+            lib.o_patch_conv_acc.restype = i64
             lib.o_epilogue.argtypes = [vp, vp, f32, vp, i32, i32, f32, vp, i64, i32]
             lib.o_f32_to_f16.argtypes = [f32]
             lib.o_f32_to_f16.restype = ctypes.c_uint16
@@ -153,6 +157,30 @@ def spgemm_acc_rows(Xq, vals, meta, rows):
     return acc
 
 
+def patch_rows(imgq, P, Kp=None):
+    """INT8 image codes [B, C, H, W] -> activation matrix [B*(H/P)*(W/P), Kp] of the patch-embedding GEMM."""
+    imgq = _c(imgq, np.int8)
+    B, C, H, W = imgq.shape
+    assert H % P == 0 and W % P == 0
+    K = C * P * P
+    Kp = K if Kp is None else Kp
+    assert Kp >= K
+    X = np.empty((B * (H // P) * (W // P), Kp), np.int8)
+    _load().o_patch_rows(_p(imgq), _p(X), B, C, H, W, P, Kp)
+    return X
+
+
+def patch_conv_acc(imgq, Wq4):
+    """The strided convolution on INT8 codes, as its definition; returns (acc [tokens, D], multiply-adds)."""
+    imgq, Wq4 = _c(imgq, np.int8), _c(Wq4, np.int8)
+    B, C, H, W = imgq.shape
+    D, C2, P, P2 = Wq4.shape
+    assert C2 == C and P2 == P and H % P == 0 and W % P == 0
+    acc = np.empty((B * (H // P) * (W // P), D), np.int32)
+    macs = _load().o_patch_conv_acc(_p(imgq), _p(Wq4), _p(acc), B, C, H, W, P, D)
+    return acc, int(macs)
+
+
 _OUT_DTYPES = {0: np.float16, 1: np.int8, 2: np.int32}
 
 
@@ -204,3 +232,29 @@ def layer_forward(X, prep, bias=None, act=0, out_type=0, out_scale=1.0, x_scale=
         acc = spgemm_acc_rows(Xq, prep["vals"], prep["meta"], rows)
     Y = epilogue(acc, prep["w_scale"], xs, bias, act, out_type, out_scale)
     return {"Xq": Xq, "x_scale": xs, "acc": acc, "Y": Y}
+
+
+def patch_embed_weight(W4, Kp=None):
+    """Conv weight [D, C, P, P] -> flattened [D, Kp] (zero columns beyond C*P*P), then the offline steps."""
+    W4 = _c(W4, np.float32)
+    D = W4.shape[0]
+    K = W4[0].size
+    Kp = K if Kp is None else Kp
+    Wf = np.zeros((D, Kp), np.float32)
+    Wf[:, :K] = W4.reshape(D, K)
+    return prepare_weight(Wf)
+
+
+def patch_embed_forward(img, prep, P, bias=None, out_type=0, out_scale=1.0, x_scale=None, rows=None):
+    """Patch embedding (Sec. 3.3): quantise the image, cut it into patch rows, sparse GEMM, epilogue."""
+    img = _c(img, np.float16)
+    Kp = prep["Wq"].shape[1]
+    imgq, xs = quant_act(img.reshape(1, -1), x_scale)
+    imgq = imgq.reshape(img.shape)
+    Xq = patch_rows(imgq, P, Kp)
+    if rows is None:
+        acc = spgemm_acc(Xq, prep["vals"], prep["meta"])
+    else:
+        acc = spgemm_acc_rows(Xq, prep["vals"], prep["meta"], rows)
+    Y = epilogue(acc, prep["w_scale"], xs, bias, 0, out_type, out_scale)
+    return {"imgq": imgq, "Xq": Xq, "x_scale": xs, "acc": acc, "Y": Y}

@@ -119,3 +119,61 @@ def random_layer(seed: int, M: int, N: int, K: int, x_dist: str = "normal") -> d
 
 def config_names() -> List[str]:
     return list(CONFIGS.keys())
+
+
+# ---- patch embedding (Sec. 3.3): an image batch and a convolution weight with kernel = stride = P ----
+
+@dataclass(frozen=True)
+class PatchConfig:
+    cid: int
+    name: str
+    B: int          # images
+    C: int          # input channels
+    H: int
+    W: int
+    P: int          # patch size
+    D: int          # embedding width
+
+    @property
+    def K(self) -> int:
+        return self.C * self.P * self.P
+
+    @property
+    def Kp(self) -> int:
+        """Reduction length padded to the 16 codes the GEMM's row pitch needs."""
+        return (self.K + 15) // 16 * 16
+
+    @property
+    def tokens(self) -> int:
+        return self.B * (self.H // self.P) * (self.W // self.P)
+
+
+PATCH_CONFIGS: Dict[str, PatchConfig] = {
+    "patch16_deit_base_b64": PatchConfig(20, "DeiT-Base patch embedding 16x16, batch 64", 64, 3, 224, 224, 16, 768),
+    "patch4_swin_tiny_b32": PatchConfig(21, "Swin-Tiny patch embedding 4x4, batch 32", 32, 3, 224, 224, 4, 96),
+    "patch4_swin_base_b32": PatchConfig(22, "Swin-Base patch embedding 4x4, batch 32", 32, 3, 224, 224, 4, 128),
+    "patch14_vit_huge_b8": PatchConfig(23, "ViT-Huge patch embedding 14x14, batch 8", 8, 3, 224, 224, 14, 1280),
+}
+
+# per-channel mean and standard deviation of the usual ImageNet input normalisation
+_PIXEL_MEAN = np.array([0.485, 0.456, 0.406], np.float32)
+_PIXEL_STD = np.array([0.229, 0.224, 0.225], np.float32)
+
+
+def make_patch_inputs(cfg: PatchConfig, seed: int = 0, B: Optional[int] = None) -> dict:
+    """img f16 [B, C, H, W] (uniform pixels in [0, 1), normalised per channel), W4 f32 [D, C, P, P], bias f32 [D]."""
+    nb = cfg.B if B is None else B
+    g = _rng(seed, cfg.cid, 0, "X")
+    pix = g.random((nb, cfg.C, cfg.H, cfg.W), dtype=np.float32)
+    ch = np.arange(cfg.C) % 3
+    img = (pix - _PIXEL_MEAN[ch][None, :, None, None]) / _PIXEL_STD[ch][None, :, None, None]
+    gw = _rng(seed, cfg.cid, 0, "W")
+    W4 = (gw.standard_normal((cfg.D, cfg.C, cfg.P, cfg.P), dtype=np.float32) * np.float32(0.02)).astype(np.float32)
+    gb = _rng(seed, cfg.cid, 0, "bias")
+    bias = (gb.standard_normal((cfg.D,), dtype=np.float32) * np.float32(0.01)).astype(np.float32)
+    return {"img": img.astype(np.float16), "W4": W4, "bias": bias}
+
+
+def random_patch(seed: int, B: int, C: int, H: int, W: int, P: int, D: int) -> dict:
+    """Free-form patch-embedding shapes for edge-case tests."""
+    return make_patch_inputs(PatchConfig(2000 + (seed % 1000), "adhoc", B, C, H, W, P, D), seed)

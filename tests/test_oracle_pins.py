@@ -321,3 +321,77 @@ def test_layer_forward_composition_and_sqnr():
     rows = np.array([3, 60])
     sub = oracle.layer_forward(d["X"], prep, d["bias"], act=0, rows=rows)
     assert np.array_equal(sub["Y"], out["Y"][rows])
+
+
+# ---------------------------------------------------------------- patch embedding (Sec. 3.3)
+
+PATCH_SHAPES = [(2, 3, 8, 8, 4, 5), (1, 3, 28, 42, 14, 7), (3, 2, 32, 16, 16, 4), (2, 1, 6, 4, 2, 3)]
+
+
+def _patch_case(seed, B, C, H, W, P, D):
+    rng = np.random.default_rng(seed)
+    imgq = rng.integers(-127, 128, (B, C, H, W)).astype(np.int8)
+    Wq4 = rng.integers(-127, 128, (D, C, P, P)).astype(np.int8)
+    return imgq, Wq4
+
+
+@pytest.mark.parametrize("B,C,H,W,P,D", PATCH_SHAPES)
+def test_patch_conv_matches_library_convolution_and_paper_flop_count(B, C, H, W, P, D):
+    torch = pytest.importorskip("torch")
+    imgq, Wq4 = _patch_case(1, B, C, H, W, P, D)
+    acc, macs = oracle.patch_conv_acc(imgq, Wq4)
+    # the strided convolution of a library (exact in float64 on these integers), flattened the usual way
+    ref = torch.nn.functional.conv2d(torch.from_numpy(imgq.astype(np.float64)),
+                                     torch.from_numpy(Wq4.astype(np.float64)), stride=P)
+    ref = ref.flatten(2).transpose(1, 2).reshape(-1, D).numpy()
+    assert np.array_equal(acc.astype(np.float64), ref)
+    # Sec. 3.3: FLOPs of the patch embedding = 2 * N * C * H * W * D_embed
+    assert 2 * macs == 2 * B * C * H * W * D
+
+
+@pytest.mark.parametrize("B,C,H,W,P,D", PATCH_SHAPES)
+def test_patch_rows_times_flat_weight_is_the_convolution(B, C, H, W, P, D):
+    imgq, Wq4 = _patch_case(2, B, C, H, W, P, D)
+    K = C * P * P
+    Kp = (K + 15) // 16 * 16
+    X = oracle.patch_rows(imgq, P, Kp)
+    assert X.shape == (B * (H // P) * (W // P), Kp)      # one token per patch
+    assert not X[:, K:].any()
+    # the same rearrangement written with array axes instead of loops
+    alt = imgq.reshape(B, C, H // P, P, W // P, P).transpose(0, 2, 4, 1, 3, 5).reshape(-1, K)
+    assert np.array_equal(X[:, :K], alt)
+    acc, _ = oracle.patch_conv_acc(imgq, Wq4)
+    assert np.array_equal(X[:, :K].astype(np.int64) @ Wq4.reshape(D, K).astype(np.int64).T, acc)
+
+
+def test_patch_rows_by_hand():
+    # one 1-channel 4x4 image, 2x2 patches: tokens in reading order, each patch in reading order
+    imgq = np.arange(16, dtype=np.int8).reshape(1, 1, 4, 4)
+    X = oracle.patch_rows(imgq, 2)
+    assert X.tolist() == [[0, 1, 4, 5], [2, 3, 6, 7], [8, 9, 12, 13], [10, 11, 14, 15]]
+    # two channels: a token's row is channel 0's patch, then channel 1's
+    img2 = np.stack([imgq[0, 0], -imgq[0, 0]])[None]
+    assert oracle.patch_rows(img2, 2)[1].tolist() == [2, 3, 6, 7, -2, -3, -6, -7]
+
+
+def test_patch_embed_forward_is_the_sparse_layer_on_patch_rows():
+    d = inputs.random_patch(3, 2, 3, 28, 28, 14, 16)     # K = 588, padded to 592
+    prep = oracle.patch_embed_weight(d["W4"], 592)
+    assert prep["Wq"].shape == (16, 592) and not prep["Wq"][:, 588:].any()
+    # padding the reduction axis changes neither the kept positions nor the codes (groups of four stay aligned)
+    Wp_plain = oracle.prune24(d["W4"].reshape(16, 588))
+    assert np.array_equal(prep["Wp"][:, :588], Wp_plain)
+    assert np.array_equal(prep["Wq"][:, :588], oracle.quant_weight(Wp_plain)[0])
+    r = oracle.patch_embed_forward(d["img"], prep, 14, d["bias"])
+    # one scale for the whole image tensor, from its largest magnitude
+    assert r["x_scale"] == np.float32(np.abs(d["img"].astype(np.float32)).max() / np.float32(127.0))
+    # the accumulators are those of the convolution of the pruned, quantised weight over the image codes
+    Wq4 = prep["Wq"][:, :588].reshape(16, 3, 14, 14)
+    acc, _ = oracle.patch_conv_acc(r["imgq"], Wq4)
+    assert np.array_equal(r["acc"], acc)
+    # de-quantised output tracks the FP32 convolution of the pruned weight
+    Wp4 = prep["Wp"][:, :588].reshape(16, 3, 14, 14).astype(np.float64)
+    X = d["img"].astype(np.float64).reshape(2, 3, 2, 14, 2, 14).transpose(0, 2, 4, 1, 3, 5).reshape(-1, 588)
+    ref = X @ Wp4.reshape(16, 588).T + d["bias"].astype(np.float64)
+    err = np.abs(r["Y"].astype(np.float64) - ref)
+    assert err.max() < 0.05 * np.abs(ref).max()
