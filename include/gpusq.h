@@ -164,6 +164,35 @@ int gpusq_quant_act_static(const void *X, int8_t *Xq, float *x_scale, int scale_
                            int K, void *stream);
 
 /* ---------------------------------------------------------------------------
+ * gpusq_patch_quant -- activation side of the patch-embedding layer.
+ * Paper: Sec. 3.3 (the patch embedding is a convolution with kernel size =
+ * stride = P, executed as a GEMM whose reduction axis C*P*P carries the 2:4
+ * pattern) with the quantise node of Sec. 2.2 in front of it.  One scale for
+ * the whole image tensor, as gpusq_quant_act; the codes are written as the
+ * rows of that GEMM, so gpusq_spgemm_i8 on (Xq, the packed flattened conv
+ * weight [D, Kp]) is the convolution:
+ *   Xq[t, k] = code(img[b, c, ty*P + py, tx*P + px]),
+ *   t = (b*(H/P) + ty)*(W/P) + tx,   k = (c*P + py)*P + px,
+ *   Xq[t, k] = 0 for C*P*P <= k < Kp.
+ *   img [B, C, H, W] f16 in;  Xq [B*(H/P)*(W/P), Kp] i8 out;
+ *   x_scale device float[1], written (GPUSQ_SCALE_COMPUTE) or read (_GIVEN).
+ *   Kp: row length of Xq, >= C*P*P, a multiple of 16 (the GEMM's K); the conv
+ *     weight is flattened to [D, C*P*P] row-major and padded with zero
+ *     columns to Kp before gpusq_prune24.
+ *   workspace: GPUSQ_SCALE_COMPUTE only, >= gpusq_quant_act_workspace(tokens,
+ *     Kp) bytes, 16-byte aligned; contents on entry are ignored and the words
+ *     gpusq_quant_act keeps zero are not touched, so one array serves both.
+ * Two launches (maximum, then quantise and rearrange) with the scale
+ * computed, one with the scale supplied.
+ * Requires H % P == 0, W % P == 0, P even, B*C*H*W % 8 == 0, img / Xq
+ * 16-byte aligned, and tokens * Kp / v < 2^31 with v = 8, 4 or 2, the largest
+ * of them that divides P (GPUSQ_ERR_TOO_LARGE otherwise).
+ */
+int gpusq_patch_quant(const void *img, int8_t *Xq, float *x_scale, int scale_mode, int B, int C,
+                      int H, int W, int P, int Kp, void *workspace, size_t workspace_bytes,
+                      void *stream);
+
+/* ---------------------------------------------------------------------------
  * gpusq_spgemm_i8 -- the fused layer: 2:4-sparse INT8 GEMM + epilogue.
  * Paper: Fig. 1 and Sec. 3.1 (sparse x dense = dense on the sparse tensor
  * cores, same result matrix as the dense GEMM); Sec. 2.2 (de-quantise node).

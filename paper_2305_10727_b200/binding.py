@@ -24,7 +24,7 @@ SCALE_COMPUTE, SCALE_GIVEN = 0, 1
 EXPORTS = (
     "gpusq_status_string", "gpusq_prune24", "gpusq_quant_weight", "gpusq_compress24",
     "gpusq_decompress24", "gpusq_packed_bytes", "gpusq_pack24", "gpusq_quant_act_workspace",
-    "gpusq_quant_act", "gpusq_quant_act_static", "gpusq_spgemm_i8", "gpusq_gemm_i8_dense", "gpusq_set_block_tokens",
+    "gpusq_quant_act", "gpusq_quant_act_static", "gpusq_patch_quant", "gpusq_spgemm_i8", "gpusq_gemm_i8_dense", "gpusq_set_block_tokens",
 )
 
 _lib = None
@@ -60,6 +60,7 @@ def load() -> ctypes.CDLL:
     lib.gpusq_quant_act_workspace.restype = sz
     lib.gpusq_quant_act.argtypes = [vp, vp, vp, i32, i64, i32, vp, sz, vp]
     lib.gpusq_quant_act_static.argtypes = [vp, vp, vp, i32, i64, i32, vp]
+    lib.gpusq_patch_quant.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, vp, sz, vp]
     gemm_args = [vp, vp, vp, vp, vp, i32, i32, vp, vp, i64, i32, i32, vp, vp]
     lib.gpusq_spgemm_i8.argtypes = gemm_args
     lib.gpusq_gemm_i8_dense.argtypes = gemm_args
@@ -188,6 +189,40 @@ def quant_act_static(X: torch.Tensor, Xq: Optional[torch.Tensor] = None, x_scale
     _check(load().gpusq_quant_act_static(_ptr(X), _ptr(Xq), _ptr(x_scale), scale_mode, M, K, _stream()),
            "gpusq_quant_act_static")
     return Xq, x_scale
+
+
+def patch_quant(img: torch.Tensor, P: int, Kp: Optional[int] = None, Xq: Optional[torch.Tensor] = None,
+                x_scale: Optional[torch.Tensor] = None, scale_mode: int = SCALE_COMPUTE,
+                workspace: Optional[torch.Tensor] = None):
+    """gpusq_patch_quant: img f16 [B, C, H, W] -> (Xq i8 [B*(H/P)*(W/P), Kp], x_scale)."""
+    _dev(img, torch.float16, "img")
+    B, C, H, W = img.shape
+    if Kp is None:
+        Kp = (C * P * P + 15) // 16 * 16
+    tokens = B * (H // P) * (W // P)
+    if Xq is None:
+        Xq = torch.empty((tokens, Kp), dtype=torch.int8, device=img.device)
+    if x_scale is None:
+        if scale_mode == SCALE_GIVEN:
+            raise ValueError("scale_mode GIVEN needs x_scale")
+        x_scale = torch.empty((1,), dtype=torch.float32, device=img.device)
+    if workspace is None and scale_mode == SCALE_COMPUTE:
+        workspace = torch.zeros((quant_act_workspace(tokens, Kp),), dtype=torch.uint8, device=img.device)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(load().gpusq_patch_quant(_ptr(img), _ptr(Xq), _ptr(x_scale), scale_mode, B, C, H, W, P, Kp,
+                                    _ptr(workspace), ws_bytes, _stream()), "gpusq_patch_quant")
+    return Xq, x_scale
+
+
+def flatten_conv_weight(W4: torch.Tensor, Kp: Optional[int] = None) -> torch.Tensor:
+    """Conv weight [D, C, P, P] -> [D, Kp] f32 row-major, zero columns beyond C*P*P (a copy, no arithmetic)."""
+    D = W4.shape[0]
+    K = W4[0].numel()
+    if Kp is None:
+        Kp = (K + 15) // 16 * 16
+    Wf = torch.zeros((D, Kp), dtype=torch.float32, device=W4.device)
+    Wf[:, :K] = W4.reshape(D, K)
+    return Wf
 
 
 _OUT_DTYPE = {OUT_F16: torch.float16, OUT_I8: torch.int8, OUT_I32: torch.int32}

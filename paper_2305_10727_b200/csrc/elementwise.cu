@@ -319,6 +319,78 @@ act_quant_kernel(const uint4 *__restrict__ X, uint2 *__restrict__ Xq, float *x_s
     for (; i < vec8; i += stride) Xq[i] = quant8_f16<true>(__ldg(X + i), a);
 }
 
+// ---- patch embedding (Sec. 3.3): quantise an image batch and lay it out as the GEMM's rows ----
+// The convolution with kernel = stride = P is the GEMM of patch rows with the flattened weight.
+// Xq[t, k] = code(img[b, c, ty P + py, tx P + px]) with t = (b, ty, tx) and k = (c P + py) P + px;
+// columns K .. Kp-1 are written as zeros.  A thread makes kVec neighbouring codes of one row: kVec
+// divides P and W, so they are kVec neighbouring pixels of one patch row, loaded with one aligned
+// vector load.  Consecutive threads write consecutive bytes of Xq; the reads are 2 kVec-byte pieces
+// whose 32-byte sectors are shared by the threads of neighbouring patches.
+struct PatchGeom {
+    int C, H, W, P;
+    int Tx, T;      // patches per image row, per image
+    int K, Kp;      // C P P, and the padded row length of Xq
+};
+
+template <int kVec>
+__global__ void __launch_bounds__(kThreads)
+patch_quant_kernel(const __half *__restrict__ img, int8_t *__restrict__ Xq, float *x_scale,
+                   const uint32_t *__restrict__ partial, int n_partials, const PatchGeom g, uint32_t items)
+{
+    __shared__ float red[kThreads / 32];
+    float s;
+    if (n_partials > 0) {
+        uint32_t m = 0;
+        for (int i = threadIdx.x; i < n_partials; i += blockDim.x) m = max(m, __ldg(partial + i));
+        const uint32_t bits = (uint32_t)block_max((float)m, red);
+        s = scale_from_amax(__half2float(__ushort_as_half((unsigned short)bits)));
+        if (blockIdx.x == 0 && threadIdx.x == 0) *x_scale = s;
+    } else {
+        s = *x_scale;
+    }
+    const QuantScale a = make_quant_scale(s);
+    const uint32_t per_row = (uint32_t)g.Kp / kVec, pp = (uint32_t)(g.P * g.P);
+    const uint32_t stride = gridDim.x * blockDim.x;
+    for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < items; i += stride) {
+        const uint32_t t = i / per_row;
+        const uint32_t k0 = (i - t * per_row) * kVec;
+        int8_t *dst = Xq + (int64_t)t * g.Kp + k0;
+        uint32_t lo = 0, hi = 0;                            // the kVec codes, lowest byte first
+        if (k0 < (uint32_t)g.K) {
+            const uint32_t c = k0 / pp, rem = k0 - c * pp;
+            const uint32_t py = rem / (uint32_t)g.P, px = rem - py * (uint32_t)g.P;
+            const uint32_t b = t / (uint32_t)g.T, r = t - b * (uint32_t)g.T;
+            const uint32_t ty = r / (uint32_t)g.Tx, tx = r - ty * (uint32_t)g.Tx;
+            const __half *src = img + (((int64_t)b * g.C + c) * g.H + (ty * g.P + py)) * g.W + (tx * g.P + px);
+            if (kVec == 8) {
+                const uint2 q = quant8_f16<true>(__ldg(reinterpret_cast<const uint4 *>(src)), a);
+                lo = q.x;
+                hi = q.y;
+            } else {
+                uint32_t differ = 0;
+                uint32_t h01, h23 = 0;
+                if (kVec == 4) {
+                    const uint2 v = __ldg(reinterpret_cast<const uint2 *>(src));
+                    h01 = v.x;
+                    h23 = v.y;
+                } else {
+                    h01 = __ldg(reinterpret_cast<const uint32_t *>(src));
+                }
+                const float2 f0 = h2f(h01), f1 = h2f(h23);
+                float2 m0 = quant2_sums<true>(f0, a, differ), m1 = quant2_sums<true>(f1, a, differ);
+                if (differ != 0u || a.always_divide) {
+                    m0 = quant2_exact<true>(f0, a);
+                    m1 = quant2_exact<true>(f1, a);
+                }
+                lo = pack4_low_bytes(m0, m1);
+            }
+        }
+        if (kVec == 8) *reinterpret_cast<uint2 *>(dst) = make_uint2(lo, hi);
+        else if (kVec == 4) *reinterpret_cast<uint32_t *>(dst) = lo;
+        else *reinterpret_cast<uint16_t *>(dst) = (uint16_t)lo;
+    }
+}
+
 // ---- one-launch activation quantisation (scale computed from the tensor) ----
 // A cooperative grid of one 1024-thread CTA per SM.  Each CTA owns a contiguous slice of X:
 //   1. reads it once from HBM, keeps as much of it as fits in shared memory, finds max|x|;
@@ -622,6 +694,53 @@ int gpusq_quant_act_static(const void *X, int8_t *Xq, float *x_scale, int scale_
     }
     act_quant_kernel<<<grid_for(ceil_div(vec8, 2), 8), kThreads, 0, s>>>(
         reinterpret_cast<const uint4 *>(X), reinterpret_cast<uint2 *>(Xq), x_scale, scratch, n_partials, vec8);
+    return launch_status();
+}
+
+int gpusq_patch_quant(const void *img, int8_t *Xq, float *x_scale, int scale_mode, int B, int C, int H, int W,
+                      int P, int Kp, void *workspace, size_t ws_bytes, void *stream)
+{
+    if (!img || !Xq || !x_scale) return GPUSQ_ERR_NULL;
+    if (B <= 0 || C <= 0 || H <= 0 || W <= 0 || P <= 0 || Kp <= 0) return GPUSQ_ERR_SHAPE;
+    if (H % P || W % P || P % 2 || Kp % 16) return GPUSQ_ERR_SHAPE;
+    const int64_t K = (int64_t)C * P * P;
+    const int64_t elems = (int64_t)B * C * H * W;
+    if (K > Kp || elems % 8) return GPUSQ_ERR_SHAPE;
+    if (scale_mode != GPUSQ_SCALE_COMPUTE && scale_mode != GPUSQ_SCALE_GIVEN) return GPUSQ_ERR_ARG;
+    const int vec = (P % 8 == 0) ? 8 : (P % 4 == 0) ? 4 : 2;          // W % P == 0, so vec divides W too
+    const int64_t tokens = (int64_t)B * (H / P) * (W / P);
+    const int64_t items = tokens * (Kp / vec);
+    if (items > 0x7FFFFFFF) return GPUSQ_ERR_TOO_LARGE;               // the kernel indexes its items with 32 bits
+    if (!aligned(img, 16) || !aligned(Xq, 16)) return GPUSQ_ERR_ALIGN;
+    if (scale_mode == GPUSQ_SCALE_COMPUTE) {
+        if (!workspace || ws_bytes < gpusq_quant_act_workspace(tokens, Kp)) return GPUSQ_ERR_WORKSPACE;
+        if (!aligned(workspace, 16)) return GPUSQ_ERR_ALIGN;
+    }
+    if (int st = check_arch()) return st;
+    cudaStream_t s = (cudaStream_t)stream;
+    uint32_t *partial = reinterpret_cast<uint32_t *>(workspace);
+    int n_partials = 0;
+    if (scale_mode == GPUSQ_SCALE_COMPUTE) {
+        // the partial maxima use the first words of the workspace, every one written before it is
+        // read; the words behind them (gpusq_quant_act's barrier) are not touched
+        const int64_t vec8 = elems / 8;
+        n_partials = grid_for(ceil_div(vec8, 4), 8);
+        if (n_partials > kMaxPartials) n_partials = kMaxPartials;
+        act_absmax_kernel<<<n_partials, kThreads, 0, s>>>(reinterpret_cast<const uint4 *>(img), partial, vec8);
+        if (int st = launch_status()) return st;
+    }
+    PatchGeom g;
+    g.C = C; g.H = H; g.W = W; g.P = P;
+    g.Tx = W / P; g.T = (H / P) * (W / P);
+    g.K = (int)K; g.Kp = Kp;
+    const int grid = grid_for(items, 8);
+    const __half *src = reinterpret_cast<const __half *>(img);
+    if (vec == 8)
+        patch_quant_kernel<8><<<grid, kThreads, 0, s>>>(src, Xq, x_scale, partial, n_partials, g, (uint32_t)items);
+    else if (vec == 4)
+        patch_quant_kernel<4><<<grid, kThreads, 0, s>>>(src, Xq, x_scale, partial, n_partials, g, (uint32_t)items);
+    else
+        patch_quant_kernel<2><<<grid, kThreads, 0, s>>>(src, Xq, x_scale, partial, n_partials, g, (uint32_t)items);
     return launch_status();
 }
 

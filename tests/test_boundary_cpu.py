@@ -71,6 +71,16 @@ def test_argument_errors_are_reported_before_any_cuda_call(lib):
     assert lib.gpusq_quant_act_static(p(a16), p(a16), p(a16), 5, 4, 8, None) == ARG
     assert lib.gpusq_quant_act_static(p(a16), p(a16), p(a16), 0, (1 << 29) + 1, 8, None) == TOO_LARGE
     assert lib.gpusq_quant_act_static(p(a16 + 8), p(a16), p(a16), 0, 4, 8, None) == ALIGN
+    pq = lib.gpusq_patch_quant
+    assert pq(p(a16), p(a16), None, 1, 1, 3, 32, 32, 16, 768, None, 0, None) == NULL
+    assert pq(p(a16), p(a16), p(a16), 1, 1, 3, 32, 30, 16, 768, None, 0, None) == SHAPE      # W % P
+    assert pq(p(a16), p(a16), p(a16), 1, 1, 3, 32, 32, 16, 752, None, 0, None) == SHAPE      # Kp < C P P
+    assert pq(p(a16), p(a16), p(a16), 1, 1, 3, 28, 28, 14, 588, None, 0, None) == SHAPE      # Kp % 16
+    assert pq(p(a16), p(a16), p(a16), 1, 1, 3, 21, 21, 7, 160, None, 0, None) == SHAPE       # odd P
+    assert pq(p(a16), p(a16), p(a16), 3, 1, 3, 32, 32, 16, 768, None, 0, None) == ARG
+    assert pq(p(a16), p(a16), p(a16), 0, 1, 3, 32, 32, 16, 768, None, 0, None) == WS
+    assert pq(p(a16 + 8), p(a16), p(a16), 1, 1, 3, 32, 32, 16, 768, None, 0, None) == ALIGN
+    assert pq(p(a16), p(a16), p(a16), 1, 1 << 20, 3, 224, 224, 2, 1 << 20, None, 0, None) == TOO_LARGE
     for fn in (lib.gpusq_spgemm_i8, lib.gpusq_gemm_i8_dense):
         ok = [p(a16), p(a16), p(a16), p(a16), None, 0, 0, None, p(a16), 8, 128, 64, None, None]
         bad = list(ok); bad[0] = None
