@@ -15,6 +15,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import statistics
 import subprocess
@@ -514,6 +515,155 @@ def run_gpusq(args, cfg):
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------------------- patch-embedding workload
+def run_patch_embed(args, pcfg):
+    """One step = gpusq_patch_quant (scale computed) + the sparse GEMM on the patch rows, FP16 out.
+
+    A step touches less than L2, so the timed loop walks over enough (image, Xq, Y) buffer sets to
+    exceed it; single GPU only (the layer runs once per image batch and shards like any other layer).
+    """
+    import torch
+
+    from paper_2305_10727_b200 import binding as B
+
+    if int(os.environ.get("WORLD_SIZE", "1")) != 1:
+        raise SystemExit("--patch is a single-GPU measurement")
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: libgpusq has no CPU fallback")
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    B.load()
+    peaks = load_peaks()
+    h = inputs.make_patch_inputs(pcfg)
+    T, K, Kp, D = pcfg.tokens, pcfg.K, pcfg.Kp, pcfg.D
+    Wf = B.flatten_conv_weight(torch.from_numpy(h["W4"]).to(dev), Kp)
+    Wq, ws = B.quant_weight(B.prune24(Wf))
+    vals, meta = B.compress24(Wq)
+    Wpk = B.pack24(vals, meta)
+    bias = torch.from_numpy(h["bias"]).to(dev)
+    img_bytes, xq_bytes, y_bytes = h["img"].size * 2, T * Kp, T * D * 2
+    step_bytes = 2 * img_bytes + 2 * xq_bytes + y_bytes          # image read twice, Xq written and read
+    nbuf = max(2, int(math.ceil(2.5 * 126e6 / (img_bytes + xq_bytes + y_bytes))))
+    img0 = torch.from_numpy(h["img"]).to(dev)
+    sets = [dict(img=img0.clone(), Xq=torch.empty((T, Kp), dtype=torch.int8, device=dev),
+                 Y=torch.empty((T, D), dtype=torch.float16, device=dev)) for _ in range(nbuf)]
+    xs = torch.empty((1,), dtype=torch.float32, device=dev)
+    wsb = torch.zeros((B.quant_act_workspace(T, Kp),), dtype=torch.uint8, device=dev)
+    status = torch.zeros(4, dtype=torch.int32, device=dev)
+
+    def quant(s, given=False):
+        if given:
+            B.patch_quant(s["img"], pcfg.P, Kp, s["Xq"], xs, scale_mode=B.SCALE_GIVEN)
+        else:
+            B.patch_quant(s["img"], pcfg.P, Kp, s["Xq"], xs, workspace=wsb)
+
+    def gemm(s):
+        B.spgemm_i8(s["Xq"], Wpk, D, ws, xs, bias, out_type=B.OUT_F16, Y=s["Y"], status_buf=status)
+
+    stream = torch.cuda.Stream()
+    torch.cuda.set_stream(stream)
+    replays = max(1, int(math.ceil(args.steps / nbuf)))
+    steps = replays * nbuf
+
+    def loop_ms(fn):
+        """Milliseconds per step of `fn(set)` run over all buffer sets, replayed from a graph."""
+        for s in sets[:2]:
+            fn(s)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for s in sets:
+                fn(s)
+        for _ in range(max(3, int(math.ceil(max(args.warmup, 3) / nbuf)))):
+            g.replay()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record(stream)
+        for _ in range(replays):
+            g.replay()
+        b.record(stream)
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / steps
+
+    sampler = ClockSampler(0)
+    sampler.start()
+    ms_step = loop_ms(lambda s: (quant(s), gemm(s)))
+    clocks = sampler.stop()
+    ms_quant = loop_ms(quant)
+    ms_quant_given = loop_ms(lambda s: quant(s, True))
+    ms_gemm = loop_ms(gemm)
+    ms_given_step = loop_ms(lambda s: (quant(s, True), gemm(s)))
+    flops = 2.0 * T * K * D                                     # Sec. 3.3: 2 N C H W D_embed
+    value = flops / (ms_step * 1e-3) / 1e12
+
+    # ---- end to end: image batch from pinned host memory in, embeddings out, every step
+    e2e = None
+    if not args.no_e2e:
+        pin_in = torch.from_numpy(h["img"]).pin_memory()
+        pin_out = torch.empty((T, D), dtype=torch.float16).pin_memory()
+        s0 = sets[0]
+
+        def e2e_step():
+            s0["img"].copy_(pin_in, non_blocking=True)
+            quant(s0)
+            gemm(s0)
+            pin_out.copy_(s0["Y"], non_blocking=True)
+
+        for _ in range(3):
+            e2e_step()
+        torch.cuda.synchronize()
+        n_e2e = 20
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(n_e2e):
+            e2e_step()
+        b.record(stream)
+        torch.cuda.synchronize()
+        ms_e2e = a.elapsed_time(b) / n_e2e
+        e2e = {"value": round(flops / (ms_e2e * 1e-3) / 1e12, 2), "unit": UNIT, "h2d_bytes_per_step": img_bytes,
+               "d2h_bytes_per_step": y_bytes, "ms_per_step": round(ms_e2e, 4), "steps": n_e2e}
+    status_host = status.cpu().tolist()
+
+    # ---- CPU baseline: the oracle on the first images of the batch
+    cpu_baseline = None
+    if not args.no_cpu_baseline:
+        import oracle
+        nb = max(1, min(pcfg.B, int(3e9 // (float(T // pcfg.B) * Kp * D))))      # about 3 G multiply-adds
+        prep = oracle.patch_embed_weight(h["W4"], Kp)
+        t0 = time.perf_counter()
+        oracle.patch_embed_forward(h["img"][:nb], prep, pcfg.P, h["bias"])
+        t_cpu = time.perf_counter() - t0
+        cpu_baseline = {"value": flops * nb / pcfg.B / t_cpu / 1e12, "unit": UNIT, "cores": 1, "kind": "oracle",
+                        "sample": "first %d of %d images (quantise + patch rows + GEMM + epilogue), %.1f s"
+                                  % (nb, pcfg.B, t_cpu)}
+
+    quant_bytes = 2 * img_bytes + xq_bytes                       # maximum pass + quantise pass
+    line = {
+        "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": 1, "steps": steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": round(ms_step, 5), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+        "config": {"workload": pcfg.name, "images": pcfg.B, "C": pcfg.C, "H": pcfg.H, "W": pcfg.W, "P": pcfg.P,
+                   "tokens": T, "K": K, "K_padded": Kp, "D": D,
+                   "step": "gpusq_patch_quant (scale computed: 2 launches) + sparse GEMM with fused epilogue, FP16 out",
+                   "launch": "graph", "l2": "the loop walks over %d buffer sets, %.0f MB" % (nbuf, nbuf * (img_bytes + xq_bytes + y_bytes) / 1e6),
+                   "parallelism": "single GPU"},
+        "roofline": {"bound": "hbm", "kernel": "act_absmax_kernel + patch_quant_kernel",
+                     "achieved": round(quant_bytes / (ms_quant * 1e-3) / 1e9, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": round(quant_bytes / (ms_quant * 1e-3) / 1e9 / peaks["hbm_gbs"], 4), "traffic": None,
+                     "peak_source": "%s copy bandwidth" % peaks["_source"],
+                     "timing": "CUDA events around %d graph replays of the two launches alone over the buffer sets" % replays,
+                     "patch_quant_us": round(ms_quant * 1e3, 2), "patch_quant_given_us": round(ms_quant_given * 1e3, 2),
+                     "gemm_us": round(ms_gemm * 1e3, 2),
+                     "gemm_tops": round(flops / (ms_gemm * 1e-3) / 1e12, 1),
+                     "step_hbm_gbs": round(step_bytes / (ms_step * 1e-3) / 1e9, 1)},
+        "cpu_baseline": cpu_baseline, "e2e": e2e, "gpu_launches": 3 * steps, "clocks": clocks,
+        "static_scale_step": {"us": round(ms_given_step * 1e3, 2), "note": "same step with a supplied image scale: 2 launches"},
+        "device_status": status_host,
+        "peaks": {k: v for k, v in peaks.items() if k in ("hbm_gbs", "bf16_tflops", "bf16_tflops_sustained", "_source")},
+    }
+    print(json.dumps(line))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -521,6 +671,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="gpusq", choices=["gpusq", "reference"])
     ap.add_argument("--config", default="deit_base_b64", choices=inputs.config_names())
+    ap.add_argument("--patch", default=None, choices=list(inputs.PATCH_CONFIGS),
+                    help="measure a patch-embedding workload instead of a block of linear layers")
     ap.add_argument("--launch", default="graph", choices=["graph", "eager"])
     ap.add_argument("--ref-rows", type=int, default=4096,
                     help="token rows per layer the CPU oracle is timed on (about 15 s of single-core work)")
@@ -530,6 +682,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     cfg = inputs.CONFIGS[args.config]
+    if args.patch is not None and args.impl == "gpusq":
+        run_patch_embed(args, inputs.PATCH_CONFIGS[args.patch])
+        return
     if args.impl == "reference":
         if int(os.environ.get("RANK", "0")) != 0:
             return

@@ -326,10 +326,35 @@ act_quant_kernel(const uint4 *__restrict__ X, uint2 *__restrict__ Xq, float *x_s
 // divides P and W, so they are kVec neighbouring pixels of one patch row, loaded with one aligned
 // vector load.  Consecutive threads write consecutive bytes of Xq; the reads are 2 kVec-byte pieces
 // whose 32-byte sectors are shared by the threads of neighbouring patches.
+// floor(n / d) for n < 2^31 as one multiply-high and a shift.  With 2^(s-1) < d <= 2^s and
+// m = ceil(2^(31+s) / d) < 2^32, m d exceeds 2^(31+s) by less than d <= 2^s, so n m / 2^(31+s) exceeds
+// n / d by less than n / 2^31 / d < 1 / d: not enough to reach the next integer.
+struct FastDiv {
+    uint32_t d, m, sh;
+};
+
+static FastDiv make_fast_div(uint32_t d)
+{
+    FastDiv f = {d, 0u, 0u};
+    if (d > 1) {
+        uint32_t s = 0;
+        while (((uint64_t)1 << s) < d) ++s;
+        f.m = (uint32_t)((((uint64_t)1 << (31 + s)) + d - 1) / d);
+        f.sh = s - 1;
+    }
+    return f;
+}
+
+__device__ __forceinline__ uint32_t fast_div(uint32_t n, const FastDiv &f)
+{
+    return f.d == 1 ? n : __umulhi(n, f.m) >> f.sh;
+}
+
 struct PatchGeom {
     int C, H, W, P;
     int Tx, T;      // patches per image row, per image
     int K, Kp;      // C P P, and the padded row length of Xq
+    FastDiv by_row, by_pp, by_p, by_t, by_tx;   // divisors Kp / kVec, P P, P, T, Tx
 };
 
 template <int kVec>
@@ -349,45 +374,63 @@ patch_quant_kernel(const __half *__restrict__ img, int8_t *__restrict__ Xq, floa
         s = *x_scale;
     }
     const QuantScale a = make_quant_scale(s);
-    const uint32_t per_row = (uint32_t)g.Kp / kVec, pp = (uint32_t)(g.P * g.P);
-    const uint32_t stride = gridDim.x * blockDim.x;
-    for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < items; i += stride) {
-        const uint32_t t = i / per_row;
-        const uint32_t k0 = (i - t * per_row) * kVec;
-        int8_t *dst = Xq + (int64_t)t * g.Kp + k0;
-        uint32_t lo = 0, hi = 0;                            // the kVec codes, lowest byte first
-        if (k0 < (uint32_t)g.K) {
-            const uint32_t c = k0 / pp, rem = k0 - c * pp;
-            const uint32_t py = rem / (uint32_t)g.P, px = rem - py * (uint32_t)g.P;
-            const uint32_t b = t / (uint32_t)g.T, r = t - b * (uint32_t)g.T;
-            const uint32_t ty = r / (uint32_t)g.Tx, tx = r - ty * (uint32_t)g.Tx;
-            const __half *src = img + (((int64_t)b * g.C + c) * g.H + (ty * g.P + py)) * g.W + (tx * g.P + px);
+    // item i -> where its codes go, and where its pixels are (nullptr in the padding columns);
+    // every dividend is below `items` < 2^31
+    auto locate = [&](uint32_t i, int8_t *&dst) -> const __half * {
+        const uint32_t t = fast_div(i, g.by_row);
+        const uint32_t k0 = (i - t * g.by_row.d) * kVec;
+        dst = Xq + (int64_t)t * g.Kp + k0;
+        if (k0 >= (uint32_t)g.K) return nullptr;
+        const uint32_t c = fast_div(k0, g.by_pp), rem = k0 - c * g.by_pp.d;
+        const uint32_t py = fast_div(rem, g.by_p), px = rem - py * g.by_p.d;
+        const uint32_t b = fast_div(t, g.by_t), r = t - b * g.by_t.d;
+        const uint32_t ty = fast_div(r, g.by_tx), tx = r - ty * g.by_tx.d;
+        return img + (((int64_t)b * g.C + c) * g.H + (ty * g.P + py)) * g.W + (tx * g.P + px);
+    };
+    auto fetch = [&](const __half *src) -> uint4 {         // kVec binary16 values, zero where there are none
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (src) {
             if (kVec == 8) {
-                const uint2 q = quant8_f16<true>(__ldg(reinterpret_cast<const uint4 *>(src)), a);
-                lo = q.x;
-                hi = q.y;
+                v = __ldg(reinterpret_cast<const uint4 *>(src));
+            } else if (kVec == 4) {
+                const uint2 h = __ldg(reinterpret_cast<const uint2 *>(src));
+                v.x = h.x;
+                v.y = h.y;
             } else {
-                uint32_t differ = 0;
-                uint32_t h01, h23 = 0;
-                if (kVec == 4) {
-                    const uint2 v = __ldg(reinterpret_cast<const uint2 *>(src));
-                    h01 = v.x;
-                    h23 = v.y;
-                } else {
-                    h01 = __ldg(reinterpret_cast<const uint32_t *>(src));
-                }
-                const float2 f0 = h2f(h01), f1 = h2f(h23);
-                float2 m0 = quant2_sums<true>(f0, a, differ), m1 = quant2_sums<true>(f1, a, differ);
-                if (differ != 0u || a.always_divide) {
-                    m0 = quant2_exact<true>(f0, a);
-                    m1 = quant2_exact<true>(f1, a);
-                }
-                lo = pack4_low_bytes(m0, m1);
+                v.x = __ldg(reinterpret_cast<const uint32_t *>(src));
             }
         }
-        if (kVec == 8) *reinterpret_cast<uint2 *>(dst) = make_uint2(lo, hi);
-        else if (kVec == 4) *reinterpret_cast<uint32_t *>(dst) = lo;
-        else *reinterpret_cast<uint16_t *>(dst) = (uint16_t)lo;
+        return v;
+    };
+    auto emit = [&](uint4 v, int8_t *dst) {                // code(0) = 0: the padding needs no special case
+        if (kVec == 8) {
+            *reinterpret_cast<uint2 *>(dst) = quant8_f16<true>(v, a);
+        } else {
+            uint32_t differ = 0;
+            const float2 f0 = h2f(v.x), f1 = h2f(v.y);
+            float2 m0 = quant2_sums<true>(f0, a, differ), m1 = quant2_sums<true>(f1, a, differ);
+            if (differ != 0u || a.always_divide) {
+                m0 = quant2_exact<true>(f0, a);
+                m1 = quant2_exact<true>(f1, a);
+            }
+            const uint32_t codes = pack4_low_bytes(m0, m1);
+            if (kVec == 4) *reinterpret_cast<uint32_t *>(dst) = codes;
+            else *reinterpret_cast<uint16_t *>(dst) = (uint16_t)codes;
+        }
+    };
+    const uint32_t stride = gridDim.x * blockDim.x;
+    uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    for (; i < items && stride < items - i; i += 2 * stride) {       // two items in flight per thread
+        int8_t *d0, *d1;
+        const __half *s0 = locate(i, d0), *s1 = locate(i + stride, d1);
+        const uint4 v0 = fetch(s0), v1 = fetch(s1);
+        emit(v0, d0);
+        emit(v1, d1);
+    }
+    if (i < items) {
+        int8_t *d0;
+        const __half *s0 = locate(i, d0);
+        emit(fetch(s0), d0);
     }
 }
 
@@ -733,6 +776,11 @@ int gpusq_patch_quant(const void *img, int8_t *Xq, float *x_scale, int scale_mod
     g.C = C; g.H = H; g.W = W; g.P = P;
     g.Tx = W / P; g.T = (H / P) * (W / P);
     g.K = (int)K; g.Kp = Kp;
+    g.by_row = make_fast_div((uint32_t)(Kp / vec));
+    g.by_pp = make_fast_div((uint32_t)(P * P));
+    g.by_p = make_fast_div((uint32_t)P);
+    g.by_t = make_fast_div((uint32_t)g.T);
+    g.by_tx = make_fast_div((uint32_t)g.Tx);
     const int grid = grid_for(items, 8);
     const __half *src = reinterpret_cast<const __half *>(img);
     if (vec == 8)

@@ -37,6 +37,8 @@ def f16_ulp_distance(a, b):
 SMALL = [
     (2, 3, 32, 32, 16, 128), (3, 3, 28, 28, 14, 40), (2, 3, 16, 24, 4, 96), (1, 3, 8, 8, 8, 8),
     (5, 1, 12, 20, 2, 16), (2, 4, 64, 32, 32, 24), (4, 3, 42, 14, 14, 1280), (1, 8, 6, 6, 6, 8),
+    # more items than one pass of the grid, and the narrower vector widths on wider images
+    (2, 3, 28, 56, 14, 16), (1, 2, 4, 16, 2, 8), (3, 3, 12, 40, 4, 48), (1300, 1, 16, 16, 16, 8),
 ]
 
 
