@@ -1,5 +1,5 @@
 """GPU parity at the full benchmark sizes, in the launch configuration bench.py
-times (automatic tile choice, persistent grid): the five workload configs,
+times (automatic tile choice, persistent grid): every workload config,
 every layer.  Weight-side stages and the activation codes are compared with the
 oracle in full; the GEMM and the epilogue are compared on sampled token rows the
 oracle computes one by one (first tile, the ragged last tile, random rows), plus
