@@ -24,4 +24,10 @@ from .oracle import (  # noqa: F401
     patch_conv_acc,
     patch_embed_weight,
     patch_embed_forward,
+    to_f16,
+    compress24_f16,
+    decompress24_f16,
+    spgemm_f16_rows,
+    epilogue_f16,
+    prepare_weight_f16,
 )

@@ -269,6 +269,90 @@ void o_epilogue(const int32_t *acc, const float *w_scale, float x_scale,
     }
 }
 
+/* ---- FP16 2:4 sparse model (the paper's M_SF) ---- */
+void o_to_f16(const float *W, uint16_t *Wh, int64_t count)
+{
+    for (int64_t i = 0; i < count; ++i) Wh[i] = o_f32_to_f16(W[i]);
+}
+
+void o_compress24_f16(const uint16_t *Wh, uint16_t *vals, uint8_t *meta, int N, int K)
+{
+    for (int n = 0; n < N; ++n) {
+        for (int g = 0; g < K / 4; ++g) {
+            const uint16_t *q = Wh + (int64_t)n * K + 4 * g;
+            double mag[4];
+            int i0, i1;
+            for (int i = 0; i < 4; ++i) mag[i] = fabs((double)o_f16_to_f32(q[i]));
+            keep_two(mag, &i0, &i1);
+            vals[(int64_t)n * (K / 2) + 2 * g] = q[i0];
+            vals[(int64_t)n * (K / 2) + 2 * g + 1] = q[i1];
+            uint8_t nib = (uint8_t)(i0 | (i1 << 2));
+            uint8_t *m = meta + (int64_t)n * (K / 8) + g / 2;
+            if (g & 1) *m = (uint8_t)((*m & 0x0F) | (nib << 4));
+            else *m = (uint8_t)((*m & 0xF0) | nib);
+        }
+    }
+}
+
+void o_decompress24_f16(const uint16_t *vals, const uint8_t *meta, uint16_t *Wh, int N, int K)
+{
+    for (int64_t i = 0; i < (int64_t)N * K; ++i) Wh[i] = 0;
+    for (int n = 0; n < N; ++n) {
+        for (int g = 0; g < K / 4; ++g) {
+            uint8_t byte = meta[(int64_t)n * (K / 8) + g / 2];
+            uint8_t nib = (g & 1) ? (uint8_t)(byte >> 4) : (uint8_t)(byte & 0x0F);
+            int i0 = nib & 3, i1 = (nib >> 2) & 3;
+            Wh[(int64_t)n * K + 4 * g + i0] = vals[(int64_t)n * (K / 2) + 2 * g];
+            Wh[(int64_t)n * K + 4 * g + i1] = vals[(int64_t)n * (K / 2) + 2 * g + 1];
+        }
+    }
+}
+
+void o_spgemm_f16_rows(const uint16_t *X, const uint16_t *vals, const uint8_t *meta,
+                       const int64_t *rows, int64_t n_rows, double *acc_rows, double *mag_rows,
+                       int N, int K)
+{
+    uint16_t *Wh = (uint16_t *)malloc((size_t)N * (size_t)K * sizeof(uint16_t));
+    double *Wd = (double *)malloc((size_t)N * (size_t)K * sizeof(double));
+    if (!Wh || !Wd) {
+        free(Wh);
+        free(Wd);
+        return;
+    }
+    o_decompress24_f16(vals, meta, Wh, N, K);
+    for (int64_t i = 0; i < (int64_t)N * K; ++i) Wd[i] = (double)o_f16_to_f32(Wh[i]);
+    for (int64_t r = 0; r < n_rows; ++r) {
+        const uint16_t *xrow = X + rows[r] * K;
+        for (int n = 0; n < N; ++n) {
+            double sum = 0.0, mag = 0.0;
+            for (int k = 0; k < K; ++k) {
+                /* a product of two binary16 values has 22 significant bits: exact in binary64 */
+                double p = Wd[(int64_t)n * K + k] * (double)o_f16_to_f32(xrow[k]);
+                sum += p;
+                mag += fabs(p);
+            }
+            acc_rows[r * N + n] = sum;
+            if (mag_rows) mag_rows[r * N + n] = mag;
+        }
+    }
+    free(Wh);
+    free(Wd);
+}
+
+void o_epilogue_f16(const double *acc, const float *bias, int act, uint16_t *Y, int64_t count, int N)
+{
+    for (int64_t e = 0; e < count; ++e) {
+        int n = (int)(e % N);
+        float t = (float)acc[e];
+        float y = t + (bias ? bias[n] : 0.0f);
+        if (act == 1) {
+            double yd = (double)y;
+            y = (float)(0.5 * yd * erfc(-yd / sqrt(2.0)));
+        }
+        Y[e] = o_f32_to_f16(y);
+    }
+}
+
 double o_sqnr_db(const float *ref, const float *test, int64_t count)
 {
     double sig = 0.0, noise = 0.0;

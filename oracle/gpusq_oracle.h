@@ -112,6 +112,27 @@ void o_epilogue(const int32_t *acc, const float *w_scale, float x_scale,
                 const float *bias, int act, int out_type, float out_scale,
                 void *Y, int64_t count, int N);
 
+/* ---- FP16 2:4 sparse model: Sec. 3.1 (the compressed FP16 format, 43.75 % smaller) and Sec. 3.4
+ * (the dense model is first pruned to the 2:4 sparse floating-point model M_SF).  Readings: the pruned
+ * FP32 weight is rounded to binary16 (RNE); the two kept positions of a group are re-derived from the
+ * binary16 magnitudes with the keep-two rule; metadata nibbles as in o_compress24; the layer takes
+ * binary16 activations as they are (no quantise node) and accumulates wider than binary16. ---- */
+void o_to_f16(const float *W, uint16_t *Wh, int64_t count);
+void o_compress24_f16(const uint16_t *Wh, uint16_t *vals, uint8_t *meta, int N, int K);
+void o_decompress24_f16(const uint16_t *vals, const uint8_t *meta, uint16_t *Wh, int N, int K);
+
+/* Fig. 1 / Sec. 3.1 for FP16 operands, as the definition: acc[r, n] = sum_k W[n, k] * X[rows[r], k]
+ * with every product exact and the sum in binary64 (the exact sum to ~1e-16 of mag);
+ * mag[r, n] = sum_k |W[n, k] * X[rows[r], k]| (nullable) scales the accumulation error a
+ * narrower accumulator may make. */
+void o_spgemm_f16_rows(const uint16_t *X, const uint16_t *vals, const uint8_t *meta,
+                       const int64_t *rows, int64_t n_rows, double *acc_rows, double *mag_rows,
+                       int N, int K);
+
+/* Epilogue of the FP16 layer: t = (float)acc; y = t + bias[n] (binary32); act 1: exact-erf GELU as in
+ * o_epilogue; Y = binary16(y), RNE. */
+void o_epilogue_f16(const double *acc, const float *bias, int act, uint16_t *Y, int64_t count, int N);
+
 /* binary16 <-> binary32 conversions used above (RNE narrowing). */
 uint16_t o_f32_to_f16(float f);
 float o_f16_to_f32(uint16_t h);

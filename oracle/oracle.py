@@ -57,6 +57,14 @@ def _load():
             lib.o_patch_rows.restype = None
             lib.o_patch_conv_acc.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32]
             lib.o_patch_conv_acc.restype = i64
+            lib.o_to_f16.argtypes = [vp, vp, i64]
+            lib.o_compress24_f16.argtypes = [vp, vp, vp, i32, i32]
+            lib.o_decompress24_f16.argtypes = [vp, vp, vp, i32, i32]
+            lib.o_spgemm_f16_rows.argtypes = [vp, vp, vp, vp, i64, vp, vp, i32, i32]
+            lib.o_epilogue_f16.argtypes = [vp, vp, i32, vp, i64, i32]
+            for name in ("o_to_f16", "o_compress24_f16", "o_decompress24_f16", "o_spgemm_f16_rows",
+                         "o_epilogue_f16"):
+                getattr(lib, name).restype = None
             lib.o_epilogue.argtypes = [vp, vp, f32, vp, i32, i32, f32, vp, i64, i32]
             lib.o_f32_to_f16.argtypes = [f32]
             lib.o_f32_to_f16.restype = ctypes.c_uint16
@@ -232,6 +240,64 @@ def layer_forward(X, prep, bias=None, act=0, out_type=0, out_scale=1.0, x_scale=
         acc = spgemm_acc_rows(Xq, prep["vals"], prep["meta"], rows)
     Y = epilogue(acc, prep["w_scale"], xs, bias, act, out_type, out_scale)
     return {"Xq": Xq, "x_scale": xs, "acc": acc, "Y": Y}
+
+
+# ---- FP16 2:4 sparse model (M_SF) ----
+
+def to_f16(W):
+    W = _c(W, np.float32)
+    Wh = np.empty(W.shape, np.uint16)
+    _load().o_to_f16(_p(W), _p(Wh), W.size)
+    return Wh.view(np.float16)
+
+
+def compress24_f16(Wh):
+    Wh = _c(Wh, np.float16)
+    N, K = Wh.shape
+    assert K % 8 == 0
+    vals = np.empty((N, K // 2), np.float16)
+    meta = np.empty((N, K // 8), np.uint8)
+    _load().o_compress24_f16(_p(Wh.view(np.uint16)), _p(vals.view(np.uint16)), _p(meta), N, K)
+    return vals, meta
+
+
+def decompress24_f16(vals, meta):
+    vals, meta = _c(vals, np.float16), _c(meta, np.uint8)
+    N, K = vals.shape[0], vals.shape[1] * 2
+    Wh = np.empty((N, K), np.float16)
+    _load().o_decompress24_f16(_p(vals.view(np.uint16)), _p(meta), _p(Wh.view(np.uint16)), N, K)
+    return Wh
+
+
+def spgemm_f16_rows(X, vals, meta, rows=None):
+    """Exact sums (binary64) of the FP16 sparse layer for the given token rows, and sum |products|."""
+    X, vals, meta = _c(X, np.float16), _c(vals, np.float16), _c(meta, np.uint8)
+    M, K = X.shape
+    N = vals.shape[0]
+    assert vals.shape == (N, K // 2) and meta.shape == (N, K // 8)
+    rows = np.arange(M, dtype=np.int64) if rows is None else _c(rows, np.int64)
+    acc = np.empty((rows.size, N), np.float64)
+    mag = np.empty((rows.size, N), np.float64)
+    _load().o_spgemm_f16_rows(_p(X.view(np.uint16)), _p(vals.view(np.uint16)), _p(meta), _p(rows), rows.size,
+                              _p(acc), _p(mag), N, K)
+    return acc, mag
+
+
+def epilogue_f16(acc, bias=None, act=0):
+    acc = _c(acc, np.float64)
+    if bias is not None:
+        bias = _c(bias, np.float32)
+    Y = np.empty(acc.shape, np.float16)
+    _load().o_epilogue_f16(_p(acc), _p(bias), act, _p(Y.view(np.uint16)), acc.size, acc.shape[-1])
+    return Y
+
+
+def prepare_weight_f16(W):
+    """Offline steps of the FP16 sparse model: prune -> round to binary16 -> compress."""
+    Wp, mask = prune24(W, return_mask=True)
+    Wh = to_f16(Wp)
+    vals, meta = compress24_f16(Wh)
+    return {"Wp": Wp, "mask": mask, "Wh": Wh, "vals": vals, "meta": meta}
 
 
 def patch_embed_weight(W4, Kp=None):

@@ -395,3 +395,63 @@ def test_patch_embed_forward_is_the_sparse_layer_on_patch_rows():
     ref = X @ Wp4.reshape(16, 588).T + d["bias"].astype(np.float64)
     err = np.abs(r["Y"].astype(np.float64) - ref)
     assert err.max() < 0.05 * np.abs(ref).max()
+
+
+# ---------------------------------------------------------------- FP16 2:4 sparse model (M_SF)
+
+def test_f16_storage_saving_matches_paper():
+    # Sec. 3.1: the compressed FP16 operand is 43.75 % smaller than the dense FP16 one
+    W = np.random.default_rng(0).standard_normal((64, 256)).astype(np.float32)
+    prep = oracle.prepare_weight_f16(W)
+    dense_bytes = W.size * 2
+    assert Fraction(prep["vals"].nbytes + prep["meta"].nbytes, dense_bytes) == 1 - Fraction(4375, 10000)
+
+
+def test_f16_compress_roundtrip_and_positions():
+    rng = np.random.default_rng(1)
+    W = rng.standard_normal((33, 64)).astype(np.float32)
+    W[0, :8] = [1e-9, -2.0, 0.0, 3.0, 5.0, 5.0, 5.0, 5.0]      # underflow to zero; a four-way tie
+    prep = oracle.prepare_weight_f16(W)
+    Wh = prep["Wh"]
+    assert np.array_equal(Wh, prep["Wp"].astype(np.float16))    # numpy's RNE narrowing
+    assert np.array_equal(oracle.decompress24_f16(prep["vals"], prep["meta"]), Wh)
+    # group 0 keeps positions 1 and 3, group 1 (all equal) the two lowest: nibbles 1|3<<2 and 0|1<<2
+    assert prep["meta"][0, 0] == (1 | (3 << 2)) | ((0 | (1 << 2)) << 4)
+    assert prep["vals"][0, :4].tolist() == [-2.0, 3.0, 5.0, 5.0]
+    # the kept positions are those of the pruning mask wherever both kept values stay non-zero in binary16
+    mask = prep["mask"]
+    for n in range(1, 33):
+        for g in range(16):
+            nib = (prep["meta"][n, g // 2] >> (4 * (g & 1))) & 0xF
+            assert (1 << (nib & 3)) | (1 << (nib >> 2)) == mask[n, g]
+
+
+@pytest.mark.parametrize("M,N,K", [(5, 7, 16), (9, 12, 64), (3, 4, 200)])
+def test_f16_spgemm_is_the_dense_product_of_the_pruned_matrix(M, N, K):
+    rng = np.random.default_rng(M + N + K)
+    W = (rng.standard_normal((N, K)) * 0.05).astype(np.float32)
+    X = rng.standard_normal((M, K)).astype(np.float16)
+    prep = oracle.prepare_weight_f16(W)
+    acc, mag = oracle.spgemm_f16_rows(X, prep["vals"], prep["meta"])
+    # exact rational arithmetic on the binary16 values
+    Wh = prep["Wh"]
+    for m in range(M):
+        for n in range(N):
+            exact = sum(Fraction(float(Wh[n, k])) * Fraction(float(X[m, k])) for k in range(K))
+            assert abs(Fraction(acc[m, n]) - exact) <= Fraction(mag[m, n]) * Fraction(1, 2 ** 48)
+    assert np.allclose(mag, np.abs(X.astype(np.float64)) @ np.abs(Wh.astype(np.float64)).T, rtol=1e-12)
+    # a row subset returns those rows
+    sub, _ = oracle.spgemm_f16_rows(X, prep["vals"], prep["meta"], np.array([M - 1, 0]))
+    assert np.array_equal(sub, acc[[M - 1, 0]])
+
+
+def test_f16_epilogue_roundings():
+    acc = np.array([[1.0 + 2.0 ** -30, -3.0, 0.1, 1e-9]], np.float64)
+    bias = np.array([2.0 ** -12, 0.5, 0.0, 0.0], np.float32)
+    Y = oracle.epilogue_f16(acc, bias, act=0)
+    # (float)acc drops the 2^-30; binary16 spacing at 1 is 2^-10, so 1 + 2^-12 rounds down to 1.0
+    assert Y[0].tolist() == [1.0, -2.5, np.float16(np.float32(0.1)), np.float16(np.float32(1e-9))]
+    G = oracle.epilogue_f16(np.array([[0.0, 1.0, -1.0, 10.0]], np.float64), None, act=1).astype(np.float64)
+    from math import erf, sqrt
+    want = [0.5 * v * (1 + erf(v / sqrt(2))) for v in (0.0, 1.0, -1.0, 10.0)]
+    assert np.allclose(G[0], want, rtol=2 ** -11, atol=0)
