@@ -47,7 +47,7 @@ typedef enum gpusq_status {
 } gpusq_status;
 
 enum { GPUSQ_ACT_NONE = 0, GPUSQ_ACT_GELU = 1 };
-enum { GPUSQ_OUT_F16 = 0, GPUSQ_OUT_I8 = 1, GPUSQ_OUT_I32 = 2 };
+enum { GPUSQ_OUT_F16 = 0, GPUSQ_OUT_I8 = 1, GPUSQ_OUT_I32 = 2, GPUSQ_OUT_F32 = 2 /* raw sums of the FP16 model */ };
 enum { GPUSQ_SCALE_COMPUTE = 0, GPUSQ_SCALE_GIVEN = 1 };
 
 /* Human-readable name of a status code (static string, never NULL). */
@@ -218,6 +218,38 @@ int gpusq_spgemm_i8(const int8_t *Xq, const void *Wpacked, const float *w_scale,
                     const float *x_scale, const float *bias, int act, int out_type,
                     const float *out_scale, void *Y, int64_t M, int N, int K, int32_t *status_buf,
                     void *stream);
+
+/* ---------------------------------------------------------------------------
+ * The FP16 2:4 sparse model.  Paper: Sec. 3.1 (the compressed FP16 operand:
+ * half of the values plus 2 bits of position per kept value, 43.75 % smaller)
+ * and Sec. 3.4 (the dense model is first pruned to the sparse floating-point
+ * model, which is then quantised); this is that intermediate model's layer.
+ *
+ * gpusq_compress24_f16: Wp [N, K] f32 in, already 2:4 (gpusq_prune24).  Each
+ *   weight is rounded to binary16 (nearest even); per group of four the two
+ *   values of largest binary16 magnitude (lower index on ties) are kept:
+ *   vals [N, K/2] f16 out, meta [N, K/8] u8 out, nibbles as gpusq_compress24.
+ *   Requires K % 8 == 0, Wp 16-byte and vals 8-byte aligned.
+ * gpusq_packed_bytes_f16 / gpusq_pack24_f16: size and contents of the opaque
+ *   operand gpusq_spgemm_f16 reads (values padded to N % 256, K % 128, then the
+ *   metadata in the tensor core's arrangement for 16-bit operands).  Wpacked
+ *   256-byte aligned.
+ * gpusq_spgemm_f16:
+ *   acc[m,n] = sum_k f16(W[n,k]) * X[m,k]     (exact products, FP32 accumulation
+ *                                              in the tensor core: order unspecified)
+ *   y        = acc + (bias ? bias[n] : 0);  act GPUSQ_ACT_GELU as gpusq_spgemm_i8
+ *   out_type GPUSQ_OUT_F16: Y f16 = round-half-even(y);
+ *            GPUSQ_OUT_F32: Y f32 = acc (bias, act ignored).
+ *   X [M, K] f16 in (no quantise node);  bias [N] f32 nullable;  Y [M, N] out;
+ *   status_buf as gpusq_spgemm_i8.
+ *   Requires M > 0, K % 8 == 0, N % 8 == 0 for GPUSQ_OUT_F16, X / Y 16-byte and
+ *   Wpacked 256-byte aligned.
+ */
+int gpusq_compress24_f16(const float *Wp, void *vals, uint8_t *meta, int N, int K, void *stream);
+size_t gpusq_packed_bytes_f16(int N, int K);
+int gpusq_pack24_f16(const void *vals, const uint8_t *meta, void *Wpacked, int N, int K, void *stream);
+int gpusq_spgemm_f16(const void *X, const void *Wpacked, const float *bias, int act, int out_type,
+                     void *Y, int64_t M, int N, int K, int32_t *status_buf, void *stream);
 
 /* ---------------------------------------------------------------------------
  * gpusq_gemm_i8_dense -- the same kernel and epilogue on the uncompressed

@@ -25,6 +25,7 @@ EXPORTS = (
     "gpusq_status_string", "gpusq_prune24", "gpusq_quant_weight", "gpusq_compress24",
     "gpusq_decompress24", "gpusq_packed_bytes", "gpusq_pack24", "gpusq_quant_act_workspace",
     "gpusq_quant_act", "gpusq_quant_act_static", "gpusq_patch_quant", "gpusq_spgemm_i8", "gpusq_gemm_i8_dense", "gpusq_set_block_tokens",
+    "gpusq_compress24_f16", "gpusq_packed_bytes_f16", "gpusq_pack24_f16", "gpusq_spgemm_f16",
 )
 
 _lib = None
@@ -65,8 +66,14 @@ def load() -> ctypes.CDLL:
     lib.gpusq_spgemm_i8.argtypes = gemm_args
     lib.gpusq_gemm_i8_dense.argtypes = gemm_args
     lib.gpusq_set_block_tokens.argtypes = [i32]
+    lib.gpusq_compress24_f16.argtypes = [vp, vp, vp, i32, i32, vp]
+    lib.gpusq_packed_bytes_f16.argtypes = [i32, i32]
+    lib.gpusq_packed_bytes_f16.restype = sz
+    lib.gpusq_pack24_f16.argtypes = [vp, vp, vp, i32, i32, vp]
+    lib.gpusq_spgemm_f16.argtypes = [vp, vp, vp, i32, i32, vp, i64, i32, i32, vp, vp]
     for name in EXPORTS:
-        if name not in ("gpusq_status_string", "gpusq_packed_bytes", "gpusq_quant_act_workspace"):
+        if name not in ("gpusq_status_string", "gpusq_packed_bytes", "gpusq_packed_bytes_f16",
+                        "gpusq_quant_act_workspace"):
             getattr(lib, name).restype = i32
     _lib = lib
     return lib
@@ -254,3 +261,41 @@ def gemm_i8_dense(Xq: torch.Tensor, Wq: torch.Tensor, w_scale=None, x_scale=None
 
 def set_block_tokens(block_t: int) -> None:
     _check(load().gpusq_set_block_tokens(block_t), "gpusq_set_block_tokens")
+
+
+# ---- FP16 2:4 sparse model ----
+OUT_F32 = 2
+
+
+def compress24_f16(Wp: torch.Tensor):
+    _dev(Wp, torch.float32, "Wp")
+    N, K = Wp.shape
+    vals = torch.empty((N, K // 2), dtype=torch.float16, device=Wp.device)
+    meta = torch.empty((N, K // 8), dtype=torch.uint8, device=Wp.device)
+    _check(load().gpusq_compress24_f16(_ptr(Wp), _ptr(vals), _ptr(meta), N, K, _stream()), "gpusq_compress24_f16")
+    return vals, meta
+
+
+def packed_bytes_f16(N: int, K: int) -> int:
+    return int(load().gpusq_packed_bytes_f16(N, K))
+
+
+def pack24_f16(vals: torch.Tensor, meta: torch.Tensor, Wpacked: Optional[torch.Tensor] = None):
+    _dev(vals, torch.float16, "vals")
+    _dev(meta, torch.uint8, "meta")
+    N, K = vals.shape[0], vals.shape[1] * 2
+    if Wpacked is None:
+        Wpacked = torch.empty((packed_bytes_f16(N, K),), dtype=torch.uint8, device=vals.device)
+    _check(load().gpusq_pack24_f16(_ptr(vals), _ptr(meta), _ptr(Wpacked), N, K, _stream()), "gpusq_pack24_f16")
+    return Wpacked
+
+
+def spgemm_f16(X: torch.Tensor, Wpacked: torch.Tensor, N: int, bias=None, act: int = ACT_NONE,
+               out_type: int = OUT_F16, Y=None, status_buf=None):
+    _dev(X, torch.float16, "X")
+    M, K = X.shape
+    if Y is None:
+        Y = torch.empty((M, N), dtype=torch.float16 if out_type == OUT_F16 else torch.float32, device=X.device)
+    _check(load().gpusq_spgemm_f16(_ptr(X), _ptr(Wpacked), _ptr(bias), act, out_type, _ptr(Y), M, N, K,
+                                   _ptr(status_buf), _stream()), "gpusq_spgemm_f16")
+    return Y

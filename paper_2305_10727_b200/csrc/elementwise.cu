@@ -240,6 +240,77 @@ pack24_kernel(const int8_t *__restrict__ vals, const uint8_t *__restrict__ meta,
     }
 }
 
+// ------------------------------------------------- FP16 2:4 sparse model (Sec. 3.1, Sec. 3.4)
+// Pruned FP32 weight -> binary16 (round to nearest even) -> the two kept values of every group of
+// four plus the metadata nibble, positions re-derived from the binary16 magnitudes with the keep-two
+// rule.  Two groups (eight weights) per thread: 32 bytes in, 8 + 1 bytes out.
+__global__ void __launch_bounds__(kThreads)
+compress24_f16_kernel(const float4 *__restrict__ Wp, uint2 *__restrict__ vals, uint8_t *__restrict__ meta,
+                      int64_t pairs)
+{
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < pairs; i += stride) {
+        uint32_t kept[2], nib[2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const float4 w = __ldg(Wp + 2 * i + h);
+            const __half q[4] = {__float2half_rn(w.x), __float2half_rn(w.y), __float2half_rn(w.z),
+                                 __float2half_rn(w.w)};
+            uint32_t bits[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) bits[j] = __half_as_ushort(q[j]);
+            // |binary16| patterns order like the magnitudes
+            const uint32_t mask = keep_two_mask(bits[0] & 0x7FFFu, bits[1] & 0x7FFFu, bits[2] & 0x7FFFu,
+                                                bits[3] & 0x7FFFu);
+            const uint32_t i0 = __ffs(mask) - 1, i1 = 31 - __clz(mask);
+            kept[h] = bits[i0] | (bits[i1] << 16);
+            nib[h] = i0 | (i1 << 2);
+        }
+        vals[i] = make_uint2(kept[0], kept[1]);
+        meta[i] = (uint8_t)(nib[0] | (nib[1] << 4));
+    }
+}
+
+// Np = N rounded up to 256, Kp = K rounded up to 128.  Values: [Np, Kp/2] binary16, zero padded.
+// Metadata: [Np/128][Kp/128] blocks of 2 KB, one per 128 rows x 128 columns of W, in the arrangement
+// the tensor core expects for 16-bit operands after a tcgen05.cp 128x128b: the byte that holds columns
+// 8 kb .. 8 kb + 7 of local row m sits at
+//   256 (m / 16) + 128 ((kb / 2) % 2) + 16 (m % 8) + 4 (kb / 4) + 2 ((m / 8) % 2) + kb % 2.
+// Padding groups get the well-formed nibble 0x4 (positions 0 and 1); their values are zero.
+__global__ void __launch_bounds__(kThreads)
+pack24_f16_kernel(const uint16_t *__restrict__ vals, const uint8_t *__restrict__ meta,
+                  uint8_t *__restrict__ packed, int N, int K, int Np, int Kp)
+{
+    const int row_chunks = Kp / 16;                       // 16-byte chunks (8 values) per padded value row
+    const int64_t val_chunks = (int64_t)Np * row_chunks;
+    const int kt = Kp / 128;
+    const int64_t meta_bytes = (int64_t)Np * (Kp / 8);
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    uint8_t *meta_out = packed + (int64_t)Np * Kp;        // Kp / 2 values of two bytes per row
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < val_chunks + meta_bytes; i += stride) {
+        if (i < val_chunks) {
+            const int n = (int)(i / row_chunks), c = (int)(i % row_chunks);
+            uint32_t w[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int v = 8 * c + 2 * j;              // K / 2 is a multiple of 4: pairs do not straddle the end
+                w[j] = (n < N && v < K / 2)
+                           ? __ldg(reinterpret_cast<const uint32_t *>(vals + (int64_t)n * (K / 2)) + v / 2) : 0u;
+            }
+            *reinterpret_cast<uint4 *>(packed + i * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+        } else {
+            const int64_t j = i - val_chunks;             // one destination byte: (tile_n, tile_k, offset)
+            const int off = (int)(j % 2048);
+            const int tk = (int)((j / 2048) % kt);
+            const int tn = (int)(j / (2048 * (int64_t)kt));
+            const int m = 16 * (off >> 8) + 8 * ((off >> 1) & 1) + ((off >> 4) & 7);
+            const int kb = 4 * ((off >> 2) & 3) + 2 * ((off >> 7) & 1) + (off & 1);
+            const int n = tn * 128 + m, byte = 16 * tk + kb;
+            meta_out[j] = (n < N && byte < K / 8) ? __ldg(meta + (int64_t)n * (K / 8) + byte) : (uint8_t)0x44;
+        }
+    }
+}
+
 // --------------------------------------------------------------- quant_act
 constexpr int kMaxPartials = 2048;   // workspace: one 32-bit partial maximum per block ...
 constexpr int kWorkspaceExtra = 64;  // ... and, behind them, the words of the grid-wide barrier (8-byte aligned)
@@ -656,6 +727,38 @@ int gpusq_pack24(const int8_t *vals, const uint8_t *meta, void *Wpacked, int N, 
     const int64_t chunks = (int64_t)Np * (Kp / 32) + (int64_t)Np * (Kp / 128);
     pack24_kernel<<<grid_for(chunks, 8), kThreads, 0, (cudaStream_t)stream>>>(
         vals, meta, reinterpret_cast<uint8_t *>(Wpacked), N, K, Np, Kp);
+    return launch_status();
+}
+
+int gpusq_compress24_f16(const float *Wp, void *vals, uint8_t *meta, int N, int K, void *stream)
+{
+    if (!Wp || !vals || !meta) return GPUSQ_ERR_NULL;
+    if (N <= 0 || K <= 0 || K % 8) return GPUSQ_ERR_SHAPE;
+    if (!aligned(Wp, 16) || !aligned(vals, 8)) return GPUSQ_ERR_ALIGN;
+    if (int st = check_arch()) return st;
+    const int64_t pairs = (int64_t)N * (K / 8);
+    compress24_f16_kernel<<<grid_for(pairs, 8), kThreads, 0, (cudaStream_t)stream>>>(
+        reinterpret_cast<const float4 *>(Wp), reinterpret_cast<uint2 *>(vals), meta, pairs);
+    return launch_status();
+}
+
+size_t gpusq_packed_bytes_f16(int N, int K)
+{
+    if (N <= 0 || K <= 0) return 0;
+    const size_t Np = (size_t)round_up(N, 256), Kp = (size_t)round_up(K, 128);
+    return Np * Kp + Np * Kp / 8;
+}
+
+int gpusq_pack24_f16(const void *vals, const uint8_t *meta, void *Wpacked, int N, int K, void *stream)
+{
+    if (!vals || !meta || !Wpacked) return GPUSQ_ERR_NULL;
+    if (N <= 0 || K <= 0 || K % 8) return GPUSQ_ERR_SHAPE;
+    if (!aligned(vals, 4) || !aligned(Wpacked, 256)) return GPUSQ_ERR_ALIGN;
+    if (int st = check_arch()) return st;
+    const int Np = round_up(N, 256), Kp = round_up(K, 128);
+    const int64_t items = (int64_t)Np * (Kp / 16) + (int64_t)Np * (Kp / 8);
+    pack24_f16_kernel<<<grid_for(items, 8), kThreads, 0, (cudaStream_t)stream>>>(
+        reinterpret_cast<const uint16_t *>(vals), meta, reinterpret_cast<uint8_t *>(Wpacked), N, K, Np, Kp);
     return launch_status();
 }
 

@@ -67,19 +67,25 @@ constexpr int kEpiBufs = 3;         // staging tiles per group
 constexpr int kEpiBufBytes = kChunkT * 128;           // [32 tokens][64 features] f16
 constexpr int kEpiBytes = kEpiGroups * kEpiBufs * kEpiBufBytes;
 
-template <bool kSparse>
+// kHalf: the FP16 2:4 sparse model (binary16 operands, FP32 accumulators) instead of INT8.  A stage
+// still covers 128 columns of W: 128 bytes of kept values per feature row, and two 128-byte-swizzled
+// activation tiles of 64 columns each, one behind the other.
+template <bool kSparse, bool kHalf = false>
 struct Cfg {
-    static constexpr int kABytes = kSparse ? kBlockF * 64 : kBlockF * 128;
-    static constexpr int kBBytes = (kMaxBlockT / 2) * 128;       // this CTA's half of the token rows
+    static_assert(kSparse || !kHalf, "the FP16 model exists only in the 2:4 sparse form");
+    static constexpr int kABytes = kHalf ? kBlockF * 128 : kSparse ? kBlockF * 64 : kBlockF * 128;
+    static constexpr int kBAtoms = kHalf ? 2 : 1;                // 128-byte-wide activation tiles per stage
+    static constexpr int kBBytes = kBAtoms * (kMaxBlockT / 2) * 128;   // this CTA's half of the token rows
     static constexpr int kMetaBytes = kSparse ? 2048 : 0;
     static constexpr int kStageBytes = kABytes + kBBytes + kMetaBytes;
-    static constexpr int kStages = kSparse ? 7 : 5;
+    static constexpr int kStages = kHalf ? 3 : kSparse ? 7 : 5;
     static constexpr int kCtlBytes = 1024;
     static constexpr int kSmemBytes = kStages * kStageBytes + kEpiBytes + kCtlBytes + 1024 /* alignment slack */;
-    static constexpr int kMmasPerStage = kSparse ? 2 : 4;
-    static constexpr int kAStepBytes = 32;                    // per MMA along K, both variants
-    static constexpr int kBStepBytes = kSparse ? 64 : 32;
-    static constexpr int kASwizzle = kSparse ? 64 : 128;
+    static constexpr int kMmasPerStage = kHalf ? 4 : kSparse ? 2 : 4;
+    static constexpr int kAStepBytes = 32;                    // per MMA along K, all variants
+    static constexpr int kBStepBytes = kHalf ? 64 : kSparse ? 64 : 32;
+    static constexpr int kASwizzle = kHalf ? 128 : kSparse ? 64 : 128;
+    static constexpr int kMetaColsPerMma = kHalf ? 1 : 2;     // 32-bit tensor-memory columns of metadata per MMA
     static_assert(kStageBytes % 1024 == 0, "stages keep the 1024-byte alignment of the swizzled tiles");
     static_assert(kStages <= 8, "eight metadata slots below the second accumulator");
     static_assert(kSmemBytes <= 232448, "shared memory per CTA");
@@ -165,6 +171,7 @@ __device__ __forceinline__ float2 gelu_pair(float2 y)
 // ahead), issue the next one, convert / scale / activate 16 values per thread, wait for a free
 // staging tile, two stmatrix, proxy fence, arrive on the tile's full barrier.  The loop is written
 // for few instructions per chunk: whatever can be precomputed or advanced incrementally is.
+template <bool kAccFloat>
 struct EpiF16 {
     const GemmParams *p;
     Ctl *ctl;
@@ -200,9 +207,11 @@ struct EpiF16 {
         for (int i = 0; i < 4; ++i)
 #pragma unroll
             for (int j = 0; j < 2; ++j) {
-                float2 y = __ffma2_rn(make_float2(__int2float_rn((int32_t)v[4 * i + 2 * j]),
-                                                  __int2float_rn((int32_t)v[4 * i + 2 * j + 1])),
-                                      sc2[j], bi2[j]);
+                // INT32 sums are converted; the FP16 model's FP32 sums are taken as they are (scale 1)
+                const float2 a = kAccFloat ? make_float2(__uint_as_float(v[4 * i + 2 * j]), __uint_as_float(v[4 * i + 2 * j + 1]))
+                                           : make_float2(__int2float_rn((int32_t)v[4 * i + 2 * j]),
+                                                         __int2float_rn((int32_t)v[4 * i + 2 * j + 1]));
+                float2 y = __ffma2_rn(a, sc2[j], bi2[j]);
                 if (kGelu) y = gelu_pair(y);
                 const __half2 hh = __floats2half2_rn(y.x, y.y);   // low = token 2(t%4), high = +1
                 pk[2 * i + j] = *reinterpret_cast<const uint32_t *>(&hh);
@@ -265,7 +274,7 @@ struct EpiF16 {
 #pragma unroll
             for (int j = 0; j < 2; ++j) {
                 const int n = n0 + nofs + 8 * j;           // N need not fill the last 128-feature block
-                ws_next[j] = (in && n < N) ? __ldg(w_scale + n) : 0.0f;
+                ws_next[j] = (in && n < N) ? (w_scale ? __ldg(w_scale + n) : 1.0f) : 0.0f;
                 bi_next[j] = (in && n < N && bias) ? __ldg(bias + n) : 0.0f;
             }
         };
@@ -456,13 +465,13 @@ struct EpiI8 {
 
 // kOut = GPUSQ_OUT_F16 / _I8 / _I32: one instantiation per output type, so that each epilogue gets its
 // own register allocation
-template <bool kSparse, int kOut>
+template <bool kSparse, int kOut, bool kHalf = false>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kNumThreads, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_e, const __grid_constant__ CUtensorMap map_y,
                const GemmParams p)
 {
-    using C = Cfg<kSparse>;
+    using C = Cfg<kSparse, kHalf>;
     extern __shared__ uint8_t smem_raw[];
     // operand tiles need 1024-byte alignment for the 128-byte swizzle; both CTAs of a pair get the same offsets
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -482,7 +491,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const int num_tiles = tiles_n * tiles_m;
     const int num_kb = (p.K + kBlockK - 1) / kBlockK;
     // bytes both CTAs together bring in per stage
-    const uint32_t stage_tx = 2u * (uint32_t)(C::kABytes + half_t * 128 + C::kMetaBytes);
+    const uint32_t stage_tx = 2u * (uint32_t)(C::kABytes + C::kBAtoms * half_t * 128 + C::kMetaBytes);
 
     auto a_smem = [&](int s) { return smem + s * C::kStageBytes; };
     auto b_smem = [&](int s) { return smem + s * C::kStageBytes + C::kABytes; };
@@ -547,8 +556,16 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     // all bytes of the stage, from both CTAs, are counted on CTA 0's barrier
                     const uint32_t bar = ptx::map_to_cta(ptx::smem_u32(&ctl->full[stage]), 0);
                     if (rank == 0) ptx::mbar_arrive_expect_tx(ptx::smem_u32(&ctl->full[stage]), stage_tx);
-                    ptx::tma_load_2d_pair(ptx::smem_u32(a_smem(stage)), &map_a, bar, kb * (kSparse ? 64 : 128), f0);
-                    ptx::tma_load_2d_pair(ptx::smem_u32(b_smem(stage)), &map_b, bar, kb * kBlockK, t0);
+                    ptx::tma_load_2d_pair(ptx::smem_u32(a_smem(stage)), &map_a, bar,
+                                          kb * (kHalf ? 128 : kSparse ? 64 : 128), f0);
+                    if (kHalf) {
+                        // 128 binary16 columns = two tiles of 128 bytes per token row
+                        ptx::tma_load_2d_pair(ptx::smem_u32(b_smem(stage)), &map_b, bar, kb * 256, t0);
+                        ptx::tma_load_2d_pair(ptx::smem_u32(b_smem(stage)) + (uint32_t)(half_t * 128), &map_b, bar,
+                                              kb * 256 + 128, t0);
+                    } else {
+                        ptx::tma_load_2d_pair(ptx::smem_u32(b_smem(stage)), &map_b, bar, kb * kBlockK, t0);
+                    }
                     if (kSparse) {
                         // 2 KB metadata block of (feature tile, k block) = 8 rows of 256 bytes
                         ptx::tma_load_2d_pair(ptx::smem_u32(m_smem(stage)), &map_e, bar, 0,
@@ -576,7 +593,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     } else if (warp == 1) {
         // ---------------------------------------------------------- MMA issuer
         if (rank == 0 && ptx::elect_one()) {
-            const uint32_t idesc = ptx::make_idesc_i8(kPairF, block_t, kSparse);
+            const uint32_t idesc = kHalf ? ptx::make_idesc_f16_sparse(kPairF, block_t) : ptx::make_idesc_i8(kPairF, block_t, kSparse);
             int stage = 0;
             uint32_t phase = 0;
             int local = 0;
@@ -608,9 +625,16 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
                     for (int k = 0; k < C::kMmasPerStage; ++k) {
                         const uint64_t ad = adesc + (uint64_t)((k * C::kAStepBytes) >> 4);
-                        const uint64_t bd = bdesc + (uint64_t)((k * C::kBStepBytes) >> 4);
+                        // FP16 model: MMAs 0, 1 read the first activation tile of the stage, 2, 3 the second
+                        const uint64_t bd = kHalf ? bdesc + (uint64_t)(((k & 1) * 64 + (k >> 1) * half_t * 128) >> 4)
+                                                  : bdesc + (uint64_t)((k * C::kBStepBytes) >> 4);
                         const uint32_t accum = (kb | k) != 0 ? 1u : 0u;
-                        if (kSparse)
+                        // 16-bit operands: one metadata column per MMA, addressed as an even column plus
+                        // the selector bit of the instruction descriptor for the odd one
+                        if (kHalf)
+                            ptx::tc_mma_sp_f16_pair(d_tmem, ad, bd, meta_t + (uint32_t)(k & ~1), idesc | (uint32_t)(k & 1),
+                                                    accum);
+                        else if (kSparse)
                             ptx::tc_mma_sp_i8_pair(d_tmem, ad, bd, meta_t + 2u * k, idesc, accum);
                         else
                             ptx::tc_mma_i8_pair(d_tmem, ad, bd, idesc, accum);
@@ -720,7 +744,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // ------------------------------------------------------------ epilogue
         const int quarter = warp & 3;                      // tensor-memory lanes [32q, 32q+32) are this warp's to read
         const int par = (warp - 2) >> 3;                   // FP16 path: which chunks, every other one
-        const float x_scale = (kOut == GPUSQ_OUT_I32) ? 1.0f : __ldg(p.x_scale);
+        const float x_scale = (kOut == GPUSQ_OUT_I32 || kHalf) ? 1.0f : __ldg(p.x_scale);
         const float out_scale = (kOut == GPUSQ_OUT_I8) ? __ldg(p.out_scale) : 1.0f;
         // the accumulators of both CTAs are released on CTA 0's barrier, where the MMA issuer waits
         const uint32_t tmem_empty0 = ptx::map_to_cta(ptx::smem_u32(&ctl->tmem_empty[0]), 0);
@@ -730,7 +754,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         int local = 0;
 
         if (kOut == GPUSQ_OUT_F16) {
-            EpiF16 e;
+            EpiF16<kHalf> e;
             e.p = &p;
             e.ctl = ctl;
             e.tmem_base = tmem_base;
@@ -894,7 +918,7 @@ static int choose_block_t(int64_t M, int tiles_n, int clusters, int K)
 }
 
 // SM pairs that can hold one cluster of this kernel each, per device (0 = unknown yet)
-template <bool kSparse>
+template <bool kSparse, bool kHalf = false>
 static int max_clusters(int sms)
 {
     static std::mutex mu;
@@ -906,9 +930,9 @@ static int max_clusters(int sms)
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)(sms & ~1), 1, 1);
         cfg.blockDim = dim3(kNumThreads, 1, 1);
-        cfg.dynamicSmemBytes = Cfg<kSparse>::kSmemBytes;
+        cfg.dynamicSmemBytes = Cfg<kSparse, kHalf>::kSmemBytes;
         int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, gemm_i8_kernel<kSparse, GPUSQ_OUT_F16>, &cfg) != cudaSuccess || n <= 0) {
+        if (cudaOccupancyMaxActiveClusters(&n, gemm_i8_kernel<kSparse, GPUSQ_OUT_F16, kHalf>, &cfg) != cudaSuccess || n <= 0) {
             (void)cudaGetLastError();
             n = sms / 2;
         }
@@ -1015,11 +1039,98 @@ static int launch_gemm(const int8_t *Xq, const void *Wsrc, const float *w_scale,
     return GPUSQ_OK;
 }
 
+// The FP16 2:4 sparse layer: binary16 activations as they are, FP32 accumulation, bias, optional GELU.
+static int launch_gemm_f16(const void *X, const void *Wpacked, const float *bias, int act, int out_type, void *Y,
+                           int64_t M, int N, int K, int32_t *status_buf, void *stream)
+{
+    using C = Cfg<true, true>;
+    if (!X || !Wpacked || !Y) return GPUSQ_ERR_NULL;
+    if ((out_type != GPUSQ_OUT_F16 && out_type != GPUSQ_OUT_F32) || act < 0 || act > 1) return GPUSQ_ERR_ARG;
+    if (M <= 0 || N <= 0 || K <= 0 || K % 8 || M > 0x7FFFFFFF) return GPUSQ_ERR_SHAPE;
+    if (out_type == GPUSQ_OUT_F16 && N % 8) return GPUSQ_ERR_SHAPE;
+    if (!aligned(X, 16) || !aligned(Wpacked, 256) || !aligned(Y, 16)) return GPUSQ_ERR_ALIGN;
+    if (int st = check_arch()) return st;
+
+    static std::once_flag attr_once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(attr_once, [] {
+        attr_err = cudaFuncSetAttribute(gemm_i8_kernel<true, GPUSQ_OUT_F16, true>,
+                                        cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+        if (attr_err == cudaSuccess)
+            attr_err = cudaFuncSetAttribute(gemm_i8_kernel<true, GPUSQ_OUT_I32, true>,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+    });
+    if (attr_err != cudaSuccess) return GPUSQ_ERR_CUDA;
+
+    const int sms = num_sms();
+    const int clusters = max_clusters<true, true>(sms);
+    if (clusters <= 0) return GPUSQ_ERR_CUDA;
+    const int tiles_n = (N + kPairF - 1) / kPairF;
+    const int block_t = choose_block_t(M, tiles_n, clusters, 2 * K);     // twice the bytes per column
+    const int Kp = round_up(K, 128), Np = round_up(N, kPairF);
+
+    // every tensor is described in bytes: kept values [Np, Kp] (Kp / 2 binary16 per row), activations
+    // [M, 2 K], metadata blocks of 2 KB as 8 rows of 256 bytes
+    CUtensorMap map_a, map_b, map_e;
+    bool ok = make_map_u8(&map_a, Wpacked, (uint64_t)Np, (uint64_t)Kp, 128, kBlockF, CU_TENSOR_MAP_SWIZZLE_128B);
+    ok = ok && make_map_u8(&map_b, X, (uint64_t)M, (uint64_t)K * 2, 128, (uint32_t)(block_t / 2),
+                           CU_TENSOR_MAP_SWIZZLE_128B);
+    const uint8_t *meta = reinterpret_cast<const uint8_t *>(Wpacked) + (size_t)Np * Kp;
+    ok = ok && make_map_u8(&map_e, meta, (uint64_t)(Np / 128) * (Kp / 128) * 8, 256, 256, 8,
+                           CU_TENSOR_MAP_SWIZZLE_NONE);
+    CUtensorMap map_y = map_b;      // placeholder unless the output is FP16
+    if (out_type == GPUSQ_OUT_F16) ok = ok && make_map_y_f16(&map_y, Y, (uint64_t)M, (uint64_t)N);
+    if (!ok) return GPUSQ_ERR_CUDA;
+
+    GemmParams p;
+    p.w_scale = nullptr;            // the epilogue's scale is 1
+    p.x_scale = nullptr;
+    p.bias = bias;
+    p.out_scale = nullptr;
+    p.Y = Y;
+    p.status = status_buf;
+    p.M = M;
+    p.N = N;
+    p.K = K;
+    p.block_t = block_t;
+    p.act = act;
+    p.out_type = out_type;
+
+    const int64_t tiles = (int64_t)tiles_n * ceil_div(M, block_t);
+    const int grid = 2 * (int)(tiles < clusters ? tiles : clusters);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid, 1, 1);
+    cfg.blockDim = dim3(kNumThreads, 1, 1);
+    cfg.dynamicSmemBytes = C::kSmemBytes;
+    cfg.stream = (cudaStream_t)stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t err;
+    if (out_type == GPUSQ_OUT_F16)
+        err = cudaLaunchKernelEx(&cfg, gemm_i8_kernel<true, GPUSQ_OUT_F16, true>, map_a, map_b, map_e, map_y, p);
+    else
+        err = cudaLaunchKernelEx(&cfg, gemm_i8_kernel<true, GPUSQ_OUT_I32, true>, map_a, map_b, map_e, map_y, p);
+    if (err != cudaSuccess) {
+        (void)cudaGetLastError();
+        return GPUSQ_ERR_CUDA;
+    }
+    return GPUSQ_OK;
+}
+
 }  // namespace gpusq
 
 using namespace gpusq;
 
 extern "C" {
+
+int gpusq_spgemm_f16(const void *X, const void *Wpacked, const float *bias, int act, int out_type, void *Y,
+                     int64_t M, int N, int K, int32_t *status_buf, void *stream)
+{
+    return launch_gemm_f16(X, Wpacked, bias, act, out_type, Y, M, N, K, status_buf, stream);
+}
 
 int gpusq_spgemm_i8(const int8_t *Xq, const void *Wpacked, const float *w_scale, const float *x_scale,
                     const float *bias, int act, int out_type, const float *out_scale, void *Y, int64_t M, int N,

@@ -283,6 +283,19 @@ __device__ __forceinline__ void tc_mma_sp_i8_pair(uint32_t d, uint64_t adesc, ui
         "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(meta_taddr)
         : "memory");
 }
+// binary16 A and B (the same type, as kind::f16 requires), FP32 accumulators, A 2:4 sparse
+__device__ __forceinline__ void tc_mma_sp_f16_pair(uint32_t d, uint64_t adesc, uint64_t bdesc, uint32_t meta_taddr,
+                                                   uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.sp.cta_group::2.kind::f16 [%0], %1, %2, [%5], %3, p;\n"
+        "}\n" ::"r"(d),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(meta_taddr)
+        : "memory");
+}
 // Wait for this thread's tensor-memory loads; the registers are operands so that no use of them
 // can be scheduled ahead of the wait.
 __device__ __forceinline__ void tmem_ld_wait_regs(uint32_t (&r)[16])
@@ -325,6 +338,12 @@ __host__ __device__ constexpr uint32_t make_idesc_i8(int mma_m, int mma_n, bool 
            | (1u << 7)                 // A: signed 8-bit
            | (1u << 10)                // B: signed 8-bit
            | ((uint32_t)(mma_n >> 3) << 17) | ((uint32_t)(mma_m >> 4) << 24);
+}
+
+// kind::f16, 2:4 sparse A: binary16 A and B (format 0), FP32 accumulators (format 1), K-major operands
+__host__ __device__ constexpr uint32_t make_idesc_f16_sparse(int mma_m, int mma_n)
+{
+    return (1u << 2) | (1u << 4) | ((uint32_t)(mma_n >> 3) << 17) | ((uint32_t)(mma_m >> 4) << 24);
 }
 
 }  // namespace ptx

@@ -103,6 +103,23 @@ def test_argument_errors_are_reported_before_any_cuda_call(lib):
         assert fn(*bad) == NULL                   # FP16 output needs w_scale
         bad = list(ok); bad[8] = p(a16 + 8)
         assert fn(*bad) == ALIGN
+    f16 = lib.gpusq_spgemm_f16
+    ok = [p(a16), p(a16), None, 0, 0, p(a16), 8, 128, 64, None, None]
+    bad = list(ok); bad[1] = None
+    assert f16(*bad) == NULL
+    bad = list(ok); bad[4] = 1
+    assert f16(*bad) == ARG                       # no INT8 output in the FP16 model
+    bad = list(ok); bad[8] = 60
+    assert f16(*bad) == SHAPE                     # K % 8
+    bad = list(ok); bad[7] = 100
+    assert f16(*bad) == SHAPE                     # FP16 rows of Y: N % 8
+    bad = list(ok); bad[0] = p(a16 + 8)
+    assert f16(*bad) == ALIGN
+    assert lib.gpusq_compress24_f16(p(a16), p(a16), None, 4, 8, None) == NULL
+    assert lib.gpusq_compress24_f16(p(a16), p(a16), p(a16), 4, 12, None) == SHAPE
+    assert lib.gpusq_pack24_f16(p(a16), p(a16), p(a16 + 16), 4, 8, None) == ALIGN
+    assert B.packed_bytes_f16(768, 768) == 768 * 768 * 9 // 8
+    assert B.packed_bytes_f16(100, 64) == 256 * 128 * 9 // 8
     assert lib.gpusq_set_block_tokens(17) == ARG
     assert lib.gpusq_set_block_tokens(256) == ARG
     assert lib.gpusq_set_block_tokens(0) == 0
