@@ -368,6 +368,29 @@ def run_gpusq(args, cfg):
                         layer_quant(s)
                         layer_gemm(s)
             ms_chain = loop_ms(step_chain)
+    # the paper's intermediate FP16 2:4 sparse model (Sec. 3.4): the same four layers on binary16
+    # weights and activations, no quantise node, FP32 accumulation: extra information
+    ms_half, half_layer_us = None, {}
+    if all(s["L"].K % 8 == 0 and s["L"].N % 8 == 0 for s in state):
+        for s in state:
+            Wt = torch.from_numpy(host[state.index(s)]["W"]).to(dev)
+            hv, hm = B.compress24_f16(B.prune24(Wt))
+            s["Wpk16"] = B.pack24_f16(hv, hm)
+            del Wt, hv, hm
+
+        def half_gemm(s):
+            B.spgemm_f16(s["X"], s["Wpk16"], s["L"].N, bias=s["bias"],
+                         act=B.ACT_GELU if s["L"].gelu else B.ACT_NONE, out_type=B.OUT_F16, Y=s["Y"], status_buf=status)
+
+        def step_half(skip=()):
+            def fn():
+                for i, s in enumerate(state):
+                    if i not in skip:
+                        half_gemm(s)
+            return fn
+        ms_half = loop_ms(step_half())
+        for i, s in enumerate(state):
+            half_layer_us[s["L"].name] = round(max(ms_half - loop_ms(step_half(skip=(i,))), 1e-3) * 1e3, 2)
     ms_dense = loop_ms(step_without(gemm=layer_gemm_dense))
     for i, s in enumerate(state):
         name = s["L"].name
@@ -507,6 +530,11 @@ def run_gpusq(args, cfg):
             "int8_chained_mlp_step": None if ms_chain is None else {
                 "block_us": round(ms_chain * 1e3, 2), "value": round(flops_step / (ms_chain * 1e-3) / 1e12, 2),
                 "unit": UNIT, "note": "fc1 writes requantised INT8 (calibrated scale) that fc2 reads: 7 launches; rank 0 only"},
+            "fp16_sparse_step": None if ms_half is None else {
+                "block_us": round(ms_half * 1e3, 2), "value": round(flops_step / (ms_half * 1e-3) / 1e12, 2),
+                "unit": "TFLOP/s (dense-equivalent)", "layers_us": half_layer_us,
+                "frac_of_measured_bf16_sustained_x2": round(flops_step / (ms_half * 1e-3) / 1e12 / (2.0 * peaks["bf16_tflops_sustained"]), 4),
+                "note": "the FP16 2:4 sparse model: four gpusq_spgemm_f16 launches on FP16 activations, no quantise node; rank 0 only"},
             "device_status": status_host, "peaks": {k: v for k, v in peaks.items() if k in ("hbm_gbs", "bf16_tflops", "bf16_tflops_sustained", "_source")},
         }
         print(json.dumps(line))
