@@ -63,7 +63,7 @@ constexpr int kTmemCols = 512;
 constexpr int kAccStride = 256;     // column offset of the second accumulator
 constexpr int kMetaCol = 224;       // metadata slots: 4 columns per stage from here (below the second accumulator)
 constexpr int kEpiGroups = 4;       // groups of four epilogue warps: 64 features x every other chunk
-constexpr int kEpiBufs = 3;         // staging tiles per group
+constexpr int kEpiBufs = 3;         // staging tiles per group (two in the FP16 model, which needs the room for a fourth stage)
 constexpr int kEpiBufBytes = kChunkT * 128;           // [32 tokens][64 features] f16
 constexpr int kEpiBytes = kEpiGroups * kEpiBufs * kEpiBufBytes;
 
@@ -78,7 +78,9 @@ struct Cfg {
     static constexpr int kBBytes = kBAtoms * (kMaxBlockT / 2) * 128;   // this CTA's half of the token rows
     static constexpr int kMetaBytes = kSparse ? 2048 : 0;
     static constexpr int kStageBytes = kABytes + kBBytes + kMetaBytes;
-    static constexpr int kStages = kHalf ? 3 : kSparse ? 7 : 5;
+    static constexpr int kStages = kHalf ? 4 : kSparse ? 7 : 5;
+    static constexpr int kEpiBufs = kHalf ? 2 : gpusq::kEpiBufs;
+    static constexpr int kEpiBytes = kEpiGroups * kEpiBufs * kEpiBufBytes;
     static constexpr int kCtlBytes = 1024;
     static constexpr int kSmemBytes = kStages * kStageBytes + kEpiBytes + kCtlBytes + 1024 /* alignment slack */;
     static constexpr int kMmasPerStage = kHalf ? 4 : kSparse ? 2 : 4;
@@ -171,7 +173,7 @@ __device__ __forceinline__ float2 gelu_pair(float2 y)
 // ahead), issue the next one, convert / scale / activate 16 values per thread, wait for a free
 // staging tile, two stmatrix, proxy fence, arrive on the tile's full barrier.  The loop is written
 // for few instructions per chunk: whatever can be precomputed or advanced incrementally is.
-template <bool kAccFloat>
+template <bool kAccFloat, int kBufs>
 struct EpiF16 {
     const GemmParams *p;
     Ctl *ctl;
@@ -228,7 +230,7 @@ struct EpiF16 {
         ptx::fence_proxy_async_smem();                     // this lane's writes, for the TMA store
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(full_bar);
-        if (++buf_idx == (uint32_t)kEpiBufs) {
+        if (++buf_idx == (uint32_t)kBufs) {
             buf_idx = 0;
             free_parity ^= 1u;
             buf_addr = stage0;
@@ -476,7 +478,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     // operand tiles need 1024-byte alignment for the 128-byte swizzle; both CTAs of a pair get the same offsets
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t *epi_smem = smem + C::kStages * C::kStageBytes;
-    Ctl *ctl = reinterpret_cast<Ctl *>(epi_smem + kEpiBytes);
+    Ctl *ctl = reinterpret_cast<Ctl *>(epi_smem + C::kEpiBytes);
+    constexpr int kBufs = C::kEpiBufs;      // staging tiles per group in the FP16-output path
     volatile uint32_t *abort_flag = &ctl->abort_flag;
 
     const int warp = threadIdx.x >> 5;
@@ -508,7 +511,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
         ptx::mbar_init(ptx::smem_u32(&ctl->drain), 1);
         for (int g = 0; g < kEpiGroups; ++g)
-            for (int b = 0; b < kEpiBufs; ++b) {
+            for (int b = 0; b < gpusq::kEpiBufs; ++b) {
                 ptx::mbar_init(ptx::smem_u32(&ctl->stg_full[g][b]), 4);
                 ptx::mbar_init(ptx::smem_u32(&ctl->stg_free[g][b]), 1);
             }
@@ -678,15 +681,15 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     const int par = (c + local) & 1;       // the group of warps that fills this chunk
                     const int gi = fgroup * 2 + par;
                     const uint32_t count = par ? filled1 : filled0;
-                    const uint32_t b = count % kEpiBufs;
+                    const uint32_t b = count % kBufs;
                     bool to;
-                    if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->stg_full[gi][b]), (count / kEpiBufs) & 1u,
+                    if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->stg_full[gi][b]), (count / kBufs) & 1u,
                                                 abort_flag, to)) {
                         if (to) report_timeout(p, ctl, tile, 3, gi * 8 + (int)b);
                         ok = false;
                         break;
                     }
-                    ptx::tma_store_2d(&map_y, ptx::smem_u32(epi_smem + (gi * kEpiBufs + (int)b) * kEpiBufBytes),
+                    ptx::tma_store_2d(&map_y, ptx::smem_u32(epi_smem + (gi * kBufs + (int)b) * kEpiBufBytes),
                                       n0 + fgroup * 64, (int32_t)(m0 + c * kChunkT));
                     ptx::tma_store_commit();
                     // all but the two newest stores have read their tiles: hand the third newest back
@@ -750,11 +753,11 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const uint32_t tmem_empty0 = ptx::map_to_cta(ptx::smem_u32(&ctl->tmem_empty[0]), 0);
         const uint32_t tmem_empty1 = ptx::map_to_cta(ptx::smem_u32(&ctl->tmem_empty[1]), 0);
         const int group = (quarter >> 1) * 2 + par;        // 64 features x chunk parity: the warps sharing staging tiles
-        const uint32_t stage0 = ptx::smem_u32(epi_smem + group * kEpiBufs * kEpiBufBytes);
+        const uint32_t stage0 = ptx::smem_u32(epi_smem + group * kBufs * kEpiBufBytes);
         int local = 0;
 
         if (kOut == GPUSQ_OUT_F16) {
-            EpiF16<kHalf> e;
+            EpiF16<kHalf, kBufs> e;
             e.p = &p;
             e.ctl = ctl;
             e.tmem_base = tmem_base;
