@@ -65,7 +65,6 @@ constexpr int kMetaCol = 224;       // metadata slots: 4 columns per stage from 
 constexpr int kEpiGroups = 4;       // groups of four epilogue warps: 64 features x every other chunk
 constexpr int kEpiBufs = 3;         // staging tiles per group (two in the FP16 model, which needs the room for a fourth stage)
 constexpr int kEpiBufBytes = kChunkT * 128;           // [32 tokens][64 features] f16
-constexpr int kEpiBytes = kEpiGroups * kEpiBufs * kEpiBufBytes;
 
 // kHalf: the FP16 2:4 sparse model (binary16 operands, FP32 accumulators) instead of INT8.  A stage
 // still covers 128 columns of W: 128 bytes of kept values per feature row, and two 128-byte-swizzled
@@ -118,7 +117,27 @@ struct GemmParams {
     int block_t;
     int act;
     int out_type;
+    int twin;       // layers of at most 128 features: the two CTAs of a pair take different token tiles
+    int oob_row;    // a row coordinate beyond the weight tensor: loads from there fill with zeros
 };
+
+// Where a tile sits.  Normally a pair shares `block_t` tokens and CTA `rank` owns 128 of the pair's
+// 256 features.  A layer of at most 128 features would leave the second CTA without output, so there
+// ("twin" tiles) each CTA owns all features of its own `block_t` tokens: the pair's MMA runs over the
+// k blocks twice, first against the token tile of CTA 0 with the weights in CTA 0's shared memory and
+// zeros in CTA 1's, then against CTA 1's tokens the other way round, so each CTA's accumulator ends
+// up with W times its own tokens.
+__device__ __forceinline__ void tile_origin(const GemmParams &p, int tiles_n, int tile, int rank, int &n0, int64_t &m0)
+{
+    if (p.twin) {
+        n0 = 0;
+        m0 = ((int64_t)tile * 2 + rank) * p.block_t;
+    } else {
+        const int tn = tile % tiles_n, tm = tile / tiles_n;
+        n0 = tn * kPairF + rank * kBlockF;
+        m0 = (int64_t)tm * p.block_t;
+    }
+}
 
 // A wait of this CTA expired: raise the abort flag in both CTAs of the pair and record where.
 __device__ __forceinline__ void report_timeout(const GemmParams &p, Ctl *ctl, int tile, int role, int stage)
@@ -271,7 +290,9 @@ struct EpiF16 {
         // scale and bias of a tile are fetched one tile ahead: the loads are in flight during a whole tile
         float ws_next[2], bi_next[2];
         auto fetch = [&](int tile) {
-            const int n0 = (tile % tiles_n) * kPairF + rank * kBlockF;
+            int n0;
+            int64_t unused;
+            tile_origin(*p, tiles_n, tile, rank, n0, unused);
             const bool in = tile < num_tiles && n0 < N;
 #pragma unroll
             for (int j = 0; j < 2; ++j) {
@@ -283,11 +304,12 @@ struct EpiF16 {
         fetch(cluster_id);
         int local = 0;
         for (int tile = cluster_id; tile < num_tiles; tile += num_clusters, ++local) {
-            const int tn = tile % tiles_n, tm = tile / tiles_n;
+            int n0;
+            int64_t m0;
+            tile_origin(*p, tiles_n, tile, rank, n0, m0);
             const int acc = local & 1;
             const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
-            const int64_t m0 = (int64_t)tm * block_t;
-            const bool n_valid = tn * kPairF + rank * kBlockF < N;     // the pair's second CTA may lie past the last feature
+            const bool n_valid = n0 < N;                   // the pair's second CTA may lie past the last feature
 #pragma unroll
             for (int j = 0; j < 2; ++j) {
                 const float sc = __fmul_rn(ws_next[j], x_scale);
@@ -372,7 +394,10 @@ struct EpiI8 {
 
         float ws_next, bi_next;
         auto fetch = [&](int tile) {
-            const int n = (tile % tiles_n) * kPairF + rank * kBlockF + quarter * 32 + lane;
+            int n0;
+            int64_t unused;
+            tile_origin(*p, tiles_n, tile, rank, n0, unused);
+            const int n = n0 + quarter * 32 + lane;
             const bool in = tile < num_tiles && n < N;
             ws_next = in ? __ldg(w_scale + n) : 0.0f;
             bi_next = (in && bias) ? __ldg(bias + n) : 0.0f;
@@ -380,11 +405,12 @@ struct EpiI8 {
         fetch(cluster_id);
         int local = 0;
         for (int tile = cluster_id; tile < num_tiles; tile += num_clusters, ++local) {
-            const int tn = tile % tiles_n, tm = tile / tiles_n;
+            int n0;
+            int64_t m0;
+            tile_origin(*p, tiles_n, tile, rank, n0, m0);
             const int acc = local & 1;
             const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
-            const int64_t m0 = (int64_t)tm * block_t;
-            const bool n_valid = tn * kPairF + rank * kBlockF < N;
+            const bool n_valid = n0 < N;
             const float sc = __fmul_rn(ws_next, x_scale);
             const float2 sc2 = make_float2(sc, sc), bi2 = make_float2(bi_next, bi_next);
             fetch(tile + num_clusters);
@@ -489,10 +515,11 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const int num_clusters = gridDim.x >> 1;
     const int block_t = p.block_t;
     const int half_t = block_t >> 1;
-    const int tiles_n = (p.N + kPairF - 1) / kPairF;
-    const int tiles_m = (int)((p.M + block_t - 1) / block_t);
+    const int tiles_n = (p.N + kPairF - 1) / kPairF;          // 1 for twin tiles
+    const int tiles_m = p.twin ? (int)((p.M + 2 * block_t - 1) / (2 * block_t)) : (int)((p.M + block_t - 1) / block_t);
     const int num_tiles = tiles_n * tiles_m;
-    const int num_kb = (p.K + kBlockK - 1) / kBlockK;
+    const int k_blocks = (p.K + kBlockK - 1) / kBlockK;        // k blocks of the layer
+    const int num_kb = p.twin ? 2 * k_blocks : k_blocks;       // stages per tile
     // bytes both CTAs together bring in per stage
     const uint32_t stage_tx = 2u * (uint32_t)(C::kABytes + C::kBAtoms * half_t * 128 + C::kMetaBytes);
 
@@ -547,9 +574,14 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             bool ok = true;
             for (int tile = cluster_id; ok && tile < num_tiles; tile += num_clusters) {
                 const int tn = tile % tiles_n, tm = tile / tiles_n;
-                const int f0 = tn * kPairF + (int)rank * kBlockF;             // this CTA's first feature
-                const int t0 = tm * block_t + (int)rank * half_t;             // this CTA's first token row
-                for (int kb = 0; kb < num_kb; ++kb) {
+                for (int ks = 0; ks < num_kb; ++ks) {
+                    // twin tiles: pass `seg` of the k blocks runs against the token tile of CTA `seg`, whose
+                    // weights sit in that CTA only (the other one loads zeros from beyond the tensor)
+                    const int seg = p.twin ? ks / k_blocks : 0;
+                    const int kb = ks - seg * k_blocks;
+                    const int w0 = p.twin ? 0 : tn * kPairF + (int)rank * kBlockF;           // first weight row wanted
+                    const int f0 = (p.twin && seg != (int)rank) ? p.oob_row : w0;          // first weight row loaded
+                    const int t0 = (p.twin ? (2 * tile + seg) * block_t : tm * block_t) + (int)rank * half_t;
                     bool to;
                     if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag, to)) {
                         if (to) report_timeout(p, ctl, tile, 0, stage);
@@ -572,7 +604,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     if (kSparse) {
                         // 2 KB metadata block of (feature tile, k block) = 8 rows of 256 bytes
                         ptx::tma_load_2d_pair(ptx::smem_u32(m_smem(stage)), &map_e, bar, 0,
-                                              ((f0 / kBlockF) * num_kb + kb) * 8);
+                                              ((w0 / kBlockF) * k_blocks + kb) * 8);
                     }
                     issued |= 1u << stage;
                     last_parity = (last_parity & ~(1u << stage)) | (phase << stage);
@@ -671,9 +703,9 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             int local = 0;
             bool ok = true;
             for (int tile = cluster_id; ok && tile < num_tiles; tile += num_clusters, ++local) {
-                const int tn = tile % tiles_n, tm = tile / tiles_n;
-                const int64_t m0 = (int64_t)tm * block_t;
-                const int n0 = tn * kPairF + (int)rank * kBlockF;
+                int n0;
+                int64_t m0;
+                tile_origin(p, tiles_n, tile, (int)rank, n0, m0);
                 if (n0 >= p.N) continue;
                 const int64_t left = p.M - m0;
                 const int nchunks = left >= block_t ? chunks : (int)((left + kChunkT - 1) / kChunkT);
@@ -713,9 +745,9 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             int local = 0;
             bool ok = true;
             for (int tile = cluster_id; ok && tile < num_tiles; tile += num_clusters, ++local) {
-                const int tn = tile % tiles_n, tm = tile / tiles_n;
-                const int64_t m0 = (int64_t)tm * block_t;
-                const int n0 = tn * kPairF + (int)rank * kBlockF;
+                int n0;
+                int64_t m0;
+                tile_origin(p, tiles_n, tile, (int)rank, n0, m0);
                 if (n0 >= p.N) continue;
                 const int64_t left = p.M - m0;
                 const int nchunks = left >= block_t ? chunks : (int)((left + kChunkT - 1) / kChunkT);
@@ -805,11 +837,11 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             // raw INT32 accumulators (for bit-exact comparison): plain coalesced stores; the four warps
             // of a quarter take every fourth 16-token chunk
             for (int tile = cluster_id; tile < num_tiles; tile += num_clusters, ++local) {
-                const int tn = tile % tiles_n, tm = tile / tiles_n;
+                int n0;
+                int64_t m0;
+                tile_origin(p, tiles_n, tile, (int)rank, n0, m0);
                 const int acc = local & 1;
                 const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
-                const int64_t m0 = (int64_t)tm * block_t;
-                const int n0 = tn * kPairF + (int)rank * kBlockF;
                 const bool n_valid = n0 < p.N;
                 const int n = n0 + quarter * 32 + lane;                // this thread's output feature
                 bool to;
@@ -977,7 +1009,9 @@ static int launch_gemm(const int8_t *Xq, const void *Wsrc, const float *w_scale,
     const int clusters = max_clusters<kSparse>(sms);
     if (clusters <= 0) return GPUSQ_ERR_CUDA;
     const int tiles_n = (N + kPairF - 1) / kPairF;
-    const int block_t = choose_block_t(M, tiles_n, clusters, K);
+    // at most 128 features: the pair's two CTAs take different token tiles (see tile_origin)
+    const bool twin = N <= kBlockF && M < 0x7FFFFFFF - 4 * kMaxBlockT;
+    const int block_t = twin ? choose_block_t(ceil_div(M, 2), 1, clusters, 2 * K) : choose_block_t(M, tiles_n, clusters, K);
     const int Kp = round_up(K, 128), Np = round_up(N, kPairF);
 
     CUtensorMap map_a, map_b;
@@ -1015,8 +1049,10 @@ static int launch_gemm(const int8_t *Xq, const void *Wsrc, const float *w_scale,
     p.block_t = block_t;
     p.act = act;
     p.out_type = out_type;
+    p.twin = twin ? 1 : 0;
+    p.oob_row = Np;                 // beyond the packed rows (Np) and the plain ones (N) alike
 
-    const int64_t tiles = (int64_t)tiles_n * ceil_div(M, block_t);
+    const int64_t tiles = twin ? ceil_div(M, 2 * (int64_t)block_t) : (int64_t)tiles_n * ceil_div(M, block_t);
     const int grid = 2 * (int)(tiles < clusters ? tiles : clusters);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid, 1, 1);
@@ -1069,7 +1105,9 @@ static int launch_gemm_f16(const void *X, const void *Wpacked, const float *bias
     const int clusters = max_clusters<true, true>(sms);
     if (clusters <= 0) return GPUSQ_ERR_CUDA;
     const int tiles_n = (N + kPairF - 1) / kPairF;
-    const int block_t = choose_block_t(M, tiles_n, clusters, 2 * K);     // twice the bytes per column
+    const bool twin = N <= kBlockF && M < 0x7FFFFFFF - 4 * kMaxBlockT;
+    // twice the bytes per column
+    const int block_t = twin ? choose_block_t(ceil_div(M, 2), 1, clusters, 4 * K) : choose_block_t(M, tiles_n, clusters, 2 * K);
     const int Kp = round_up(K, 128), Np = round_up(N, kPairF);
 
     // every tensor is described in bytes: kept values [Np, Kp] (Kp / 2 binary16 per row), activations
@@ -1098,8 +1136,10 @@ static int launch_gemm_f16(const void *X, const void *Wpacked, const float *bias
     p.block_t = block_t;
     p.act = act;
     p.out_type = out_type;
+    p.twin = twin ? 1 : 0;
+    p.oob_row = Np;
 
-    const int64_t tiles = (int64_t)tiles_n * ceil_div(M, block_t);
+    const int64_t tiles = twin ? ceil_div(M, 2 * (int64_t)block_t) : (int64_t)tiles_n * ceil_div(M, block_t);
     const int grid = 2 * (int)(tiles < clusters ? tiles : clusters);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid, 1, 1);
