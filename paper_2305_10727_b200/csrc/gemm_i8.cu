@@ -117,26 +117,35 @@ struct GemmParams {
     int block_t;
     int act;
     int out_type;
-    int twin;       // layers of at most 128 features: the two CTAs of a pair take different token tiles
+    int pair_cols;  // feature columns of 256 that are worked on as ordinary pair tiles
+    int pair_tiles; // pair_cols x token tiles: tiles from here on are twin tiles of the last 128 features
+    int num_tiles;
+    int twin_n0;    // first feature of the twin column (256 pair_cols)
     int oob_row;    // a row coordinate beyond the weight tensor: loads from there fill with zeros
 };
 
 // Where a tile sits.  Normally a pair shares `block_t` tokens and CTA `rank` owns 128 of the pair's
-// 256 features.  A layer of at most 128 features would leave the second CTA without output, so there
-// ("twin" tiles) each CTA owns all features of its own `block_t` tokens: the pair's MMA runs over the
-// k blocks twice, first against the token tile of CTA 0 with the weights in CTA 0's shared memory and
-// zeros in CTA 1's, then against CTA 1's tokens the other way round, so each CTA's accumulator ends
-// up with W times its own tokens.
-__device__ __forceinline__ void tile_origin(const GemmParams &p, int tiles_n, int tile, int rank, int &n0, int64_t &m0)
+// 256 features.  When the last column of features is at most 128 wide (N mod 256 in 1..128: every
+// layer of at most 128 features, and e.g. N = 384) that would leave the second CTA without output,
+// so that column is worked on in "twin" tiles: each CTA owns the column's features of its OWN
+// `block_t` tokens, and the pair's MMA runs over the k blocks twice, first against the token tile of
+// CTA 0 with the weight block in CTA 0's shared memory and zeros in CTA 1's, then against CTA 1's
+// tokens the other way round, so each CTA's accumulator ends up with W times its own tokens.
+// Ordinary tiles come first (feature column fastest), twin tiles after them.  Returns whether the
+// tile is a twin tile.
+// kTwin = false (no twin column in this launch) compiles the test away.
+template <bool kTwin>
+__device__ __forceinline__ bool tile_origin(const GemmParams &p, int tile, int rank, int &n0, int64_t &m0)
 {
-    if (p.twin) {
-        n0 = 0;
-        m0 = ((int64_t)tile * 2 + rank) * p.block_t;
-    } else {
-        const int tn = tile % tiles_n, tm = tile / tiles_n;
-        n0 = tn * kPairF + rank * kBlockF;
-        m0 = (int64_t)tm * p.block_t;
+    if (kTwin && tile >= p.pair_tiles) {
+        n0 = p.twin_n0;
+        m0 = ((int64_t)(tile - p.pair_tiles) * 2 + rank) * p.block_t;
+        return true;
     }
+    const int tn = tile % p.pair_cols, tm = tile / p.pair_cols;
+    n0 = tn * kPairF + rank * kBlockF;
+    m0 = (int64_t)tm * p.block_t;
+    return false;
 }
 
 // A wait of this CTA expired: raise the abort flag in both CTAs of the pair and record where.
@@ -192,7 +201,7 @@ __device__ __forceinline__ float2 gelu_pair(float2 y)
 // ahead), issue the next one, convert / scale / activate 16 values per thread, wait for a free
 // staging tile, two stmatrix, proxy fence, arrive on the tile's full barrier.  The loop is written
 // for few instructions per chunk: whatever can be precomputed or advanced incrementally is.
-template <bool kAccFloat, int kBufs>
+template <bool kAccFloat, int kBufs, bool kTwin>
 struct EpiF16 {
     const GemmParams *p;
     Ctl *ctl;
@@ -292,7 +301,7 @@ struct EpiF16 {
         auto fetch = [&](int tile) {
             int n0;
             int64_t unused;
-            tile_origin(*p, tiles_n, tile, rank, n0, unused);
+            (void)tile_origin<kTwin>(*p, tile, rank, n0, unused);
             const bool in = tile < num_tiles && n0 < N;
 #pragma unroll
             for (int j = 0; j < 2; ++j) {
@@ -306,7 +315,7 @@ struct EpiF16 {
         for (int tile = cluster_id; tile < num_tiles; tile += num_clusters, ++local) {
             int n0;
             int64_t m0;
-            tile_origin(*p, tiles_n, tile, rank, n0, m0);
+            (void)tile_origin<kTwin>(*p, tile, rank, n0, m0);
             const int acc = local & 1;
             const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
             const bool n_valid = n0 < N;                   // the pair's second CTA may lie past the last feature
@@ -357,6 +366,7 @@ struct EpiF16 {
 // word; two shuffle + byte-permute steps transpose 4 x 4 bytes among four neighbouring lanes, so that
 // each lane holds four neighbouring features of one token and writes them with one 4-byte store into
 // a 128-byte-swizzled [32 tokens][128 features] staging tile that the four quarters' warps share.
+template <bool kTwin>
 struct EpiI8 {
     const GemmParams *p;
     Ctl *ctl;
@@ -396,7 +406,7 @@ struct EpiI8 {
         auto fetch = [&](int tile) {
             int n0;
             int64_t unused;
-            tile_origin(*p, tiles_n, tile, rank, n0, unused);
+            (void)tile_origin<kTwin>(*p, tile, rank, n0, unused);
             const int n = n0 + quarter * 32 + lane;
             const bool in = tile < num_tiles && n < N;
             ws_next = in ? __ldg(w_scale + n) : 0.0f;
@@ -407,7 +417,7 @@ struct EpiI8 {
         for (int tile = cluster_id; tile < num_tiles; tile += num_clusters, ++local) {
             int n0;
             int64_t m0;
-            tile_origin(*p, tiles_n, tile, rank, n0, m0);
+            (void)tile_origin<kTwin>(*p, tile, rank, n0, m0);
             const int acc = local & 1;
             const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
             const bool n_valid = n0 < N;
@@ -493,7 +503,7 @@ struct EpiI8 {
 
 // kOut = GPUSQ_OUT_F16 / _I8 / _I32: one instantiation per output type, so that each epilogue gets its
 // own register allocation
-template <bool kSparse, int kOut, bool kHalf = false>
+template <bool kSparse, int kOut, bool kHalf = false, bool kTwin = false>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kNumThreads, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_e, const __grid_constant__ CUtensorMap map_y,
@@ -515,11 +525,9 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const int num_clusters = gridDim.x >> 1;
     const int block_t = p.block_t;
     const int half_t = block_t >> 1;
-    const int tiles_n = (p.N + kPairF - 1) / kPairF;          // 1 for twin tiles
-    const int tiles_m = p.twin ? (int)((p.M + 2 * block_t - 1) / (2 * block_t)) : (int)((p.M + block_t - 1) / block_t);
-    const int num_tiles = tiles_n * tiles_m;
-    const int k_blocks = (p.K + kBlockK - 1) / kBlockK;        // k blocks of the layer
-    const int num_kb = p.twin ? 2 * k_blocks : k_blocks;       // stages per tile
+    const int tiles_n = (p.N + kPairF - 1) / kPairF;
+    const int num_tiles = p.num_tiles;
+    const int k_blocks = (p.K + kBlockK - 1) / kBlockK;        // k blocks of the layer; a twin tile takes them twice
     // bytes both CTAs together bring in per stage
     const uint32_t stage_tx = 2u * (uint32_t)(C::kABytes + C::kBAtoms * half_t * 128 + C::kMetaBytes);
 
@@ -573,15 +581,18 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             uint32_t last_parity = 0;       // bit s: parity of the last phase issued into stage s
             bool ok = true;
             for (int tile = cluster_id; ok && tile < num_tiles; tile += num_clusters) {
-                const int tn = tile % tiles_n, tm = tile / tiles_n;
+                const bool twin = kTwin && tile >= p.pair_tiles;
+                const int tw = tile - p.pair_tiles;                               // index among the twin tiles
+                const int tn = twin ? 0 : tile % p.pair_cols, tm = twin ? 0 : tile / p.pair_cols;
+                const int num_kb = twin ? 2 * k_blocks : k_blocks;
                 for (int ks = 0; ks < num_kb; ++ks) {
                     // twin tiles: pass `seg` of the k blocks runs against the token tile of CTA `seg`, whose
                     // weights sit in that CTA only (the other one loads zeros from beyond the tensor)
-                    const int seg = p.twin ? ks / k_blocks : 0;
+                    const int seg = twin ? ks / k_blocks : 0;
                     const int kb = ks - seg * k_blocks;
-                    const int w0 = p.twin ? 0 : tn * kPairF + (int)rank * kBlockF;           // first weight row wanted
-                    const int f0 = (p.twin && seg != (int)rank) ? p.oob_row : w0;          // first weight row loaded
-                    const int t0 = (p.twin ? (2 * tile + seg) * block_t : tm * block_t) + (int)rank * half_t;
+                    const int w0 = twin ? p.twin_n0 : tn * kPairF + (int)rank * kBlockF;   // first weight row wanted
+                    const int f0 = (twin && seg != (int)rank) ? p.oob_row : w0;          // first weight row loaded
+                    const int t0 = (twin ? (2 * tw + seg) * block_t : tm * block_t) + (int)rank * half_t;
                     bool to;
                     if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag, to)) {
                         if (to) report_timeout(p, ctl, tile, 0, stage);
@@ -644,6 +655,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 }
                 ptx::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kAccStride);
+                const int num_kb = (kTwin && tile >= p.pair_tiles) ? 2 * k_blocks : k_blocks;
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->full[stage]), phase, abort_flag, to)) {
                         if (to) report_timeout(p, ctl, tile, 1, stage);
@@ -705,7 +717,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             for (int tile = cluster_id; ok && tile < num_tiles; tile += num_clusters, ++local) {
                 int n0;
                 int64_t m0;
-                tile_origin(p, tiles_n, tile, (int)rank, n0, m0);
+                (void)tile_origin<kTwin>(p, tile, (int)rank, n0, m0);
                 if (n0 >= p.N) continue;
                 const int64_t left = p.M - m0;
                 const int nchunks = left >= block_t ? chunks : (int)((left + kChunkT - 1) / kChunkT);
@@ -747,7 +759,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             for (int tile = cluster_id; ok && tile < num_tiles; tile += num_clusters, ++local) {
                 int n0;
                 int64_t m0;
-                tile_origin(p, tiles_n, tile, (int)rank, n0, m0);
+                (void)tile_origin<kTwin>(p, tile, (int)rank, n0, m0);
                 if (n0 >= p.N) continue;
                 const int64_t left = p.M - m0;
                 const int nchunks = left >= block_t ? chunks : (int)((left + kChunkT - 1) / kChunkT);
@@ -789,7 +801,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         int local = 0;
 
         if (kOut == GPUSQ_OUT_F16) {
-            EpiF16<kHalf, kBufs> e;
+            EpiF16<kHalf, kBufs, kTwin> e;
             e.p = &p;
             e.ctl = ctl;
             e.tmem_base = tmem_base;
@@ -812,7 +824,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             else
                 e.template run<false>();
         } else if (kOut == GPUSQ_OUT_I8) {
-            EpiI8 e;
+            EpiI8<kTwin> e;
             e.p = &p;
             e.ctl = ctl;
             e.epi_smem = epi_smem;
@@ -839,7 +851,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             for (int tile = cluster_id; tile < num_tiles; tile += num_clusters, ++local) {
                 int n0;
                 int64_t m0;
-                tile_origin(p, tiles_n, tile, (int)rank, n0, m0);
+                (void)tile_origin<kTwin>(p, tile, (int)rank, n0, m0);
                 const int acc = local & 1;
                 const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
                 const bool n_valid = n0 < p.N;
@@ -995,13 +1007,20 @@ static int launch_gemm(const int8_t *Xq, const void *Wsrc, const float *w_scale,
     static std::once_flag attr_once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(attr_once, [] {
-        const void *kernels[6] = {
+        const void *kernels[12] = {
             (const void *)gemm_i8_kernel<true, GPUSQ_OUT_F16>,  (const void *)gemm_i8_kernel<true, GPUSQ_OUT_I8>,
-            (const void *)gemm_i8_kernel<true, GPUSQ_OUT_I32>,  (const void *)gemm_i8_kernel<false, GPUSQ_OUT_F16>,
-            (const void *)gemm_i8_kernel<false, GPUSQ_OUT_I8>,  (const void *)gemm_i8_kernel<false, GPUSQ_OUT_I32>};
-        for (int k = 0; k < 6 && attr_err == cudaSuccess; ++k)
+            (const void *)gemm_i8_kernel<true, GPUSQ_OUT_I32>,
+            (const void *)gemm_i8_kernel<true, GPUSQ_OUT_F16, false, true>,
+            (const void *)gemm_i8_kernel<true, GPUSQ_OUT_I8, false, true>,
+            (const void *)gemm_i8_kernel<true, GPUSQ_OUT_I32, false, true>,
+            (const void *)gemm_i8_kernel<false, GPUSQ_OUT_F16>, (const void *)gemm_i8_kernel<false, GPUSQ_OUT_I8>,
+            (const void *)gemm_i8_kernel<false, GPUSQ_OUT_I32>,
+            (const void *)gemm_i8_kernel<false, GPUSQ_OUT_F16, false, true>,
+            (const void *)gemm_i8_kernel<false, GPUSQ_OUT_I8, false, true>,
+            (const void *)gemm_i8_kernel<false, GPUSQ_OUT_I32, false, true>};
+        for (int k = 0; k < 12 && attr_err == cudaSuccess; ++k)
             attr_err = cudaFuncSetAttribute(kernels[k], cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            k < 3 ? Cfg<true>::kSmemBytes : Cfg<false>::kSmemBytes);
+                                            k < 6 ? Cfg<true>::kSmemBytes : Cfg<false>::kSmemBytes);
     });
     if (attr_err != cudaSuccess) return GPUSQ_ERR_CUDA;
 
@@ -1009,9 +1028,10 @@ static int launch_gemm(const int8_t *Xq, const void *Wsrc, const float *w_scale,
     const int clusters = max_clusters<kSparse>(sms);
     if (clusters <= 0) return GPUSQ_ERR_CUDA;
     const int tiles_n = (N + kPairF - 1) / kPairF;
-    // at most 128 features: the pair's two CTAs take different token tiles (see tile_origin)
-    const bool twin = N <= kBlockF && M < 0x7FFFFFFF - 4 * kMaxBlockT;
-    const int block_t = twin ? choose_block_t(ceil_div(M, 2), 1, clusters, 2 * K) : choose_block_t(M, tiles_n, clusters, K);
+    // a last feature column of at most 128 features is worked on in twin tiles (see tile_origin)
+    const bool twin_col = N - (tiles_n - 1) * kPairF <= kBlockF && M < 0x7FFFFFFF - 4 * kMaxBlockT;
+    const int block_t = (twin_col && tiles_n == 1) ? choose_block_t(ceil_div(M, 2), 1, clusters, 2 * K)
+                                                   : choose_block_t(M, tiles_n, clusters, K);
     const int Kp = round_up(K, 128), Np = round_up(N, kPairF);
 
     CUtensorMap map_a, map_b;
@@ -1049,10 +1069,15 @@ static int launch_gemm(const int8_t *Xq, const void *Wsrc, const float *w_scale,
     p.block_t = block_t;
     p.act = act;
     p.out_type = out_type;
-    p.twin = twin ? 1 : 0;
+    p.pair_cols = twin_col ? tiles_n - 1 : tiles_n;
+    const int64_t pair_tiles = (int64_t)p.pair_cols * ceil_div(M, block_t);
+    const int64_t tiles = pair_tiles + (twin_col ? ceil_div(M, 2 * (int64_t)block_t) : 0);
+    if (tiles > 0x7FFFFFFF) return GPUSQ_ERR_SHAPE;
+    p.pair_tiles = (int)pair_tiles;
+    p.num_tiles = (int)tiles;
+    p.twin_n0 = p.pair_cols * kPairF;
     p.oob_row = Np;                 // beyond the packed rows (Np) and the plain ones (N) alike
 
-    const int64_t tiles = twin ? ceil_div(M, 2 * (int64_t)block_t) : (int64_t)tiles_n * ceil_div(M, block_t);
     const int grid = 2 * (int)(tiles < clusters ? tiles : clusters);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid, 1, 1);
@@ -1065,12 +1090,16 @@ static int launch_gemm(const int8_t *Xq, const void *Wsrc, const float *w_scale,
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     cudaError_t err;
+    // launches without a twin column run the instantiation that has no trace of it
     if (out_type == GPUSQ_OUT_F16)
-        err = cudaLaunchKernelEx(&cfg, gemm_i8_kernel<kSparse, GPUSQ_OUT_F16>, map_a, map_b, map_e, map_y, p);
+        err = twin_col ? cudaLaunchKernelEx(&cfg, gemm_i8_kernel<kSparse, GPUSQ_OUT_F16, false, true>, map_a, map_b, map_e, map_y, p)
+                       : cudaLaunchKernelEx(&cfg, gemm_i8_kernel<kSparse, GPUSQ_OUT_F16>, map_a, map_b, map_e, map_y, p);
     else if (out_type == GPUSQ_OUT_I8)
-        err = cudaLaunchKernelEx(&cfg, gemm_i8_kernel<kSparse, GPUSQ_OUT_I8>, map_a, map_b, map_e, map_y, p);
+        err = twin_col ? cudaLaunchKernelEx(&cfg, gemm_i8_kernel<kSparse, GPUSQ_OUT_I8, false, true>, map_a, map_b, map_e, map_y, p)
+                       : cudaLaunchKernelEx(&cfg, gemm_i8_kernel<kSparse, GPUSQ_OUT_I8>, map_a, map_b, map_e, map_y, p);
     else
-        err = cudaLaunchKernelEx(&cfg, gemm_i8_kernel<kSparse, GPUSQ_OUT_I32>, map_a, map_b, map_e, map_y, p);
+        err = twin_col ? cudaLaunchKernelEx(&cfg, gemm_i8_kernel<kSparse, GPUSQ_OUT_I32, false, true>, map_a, map_b, map_e, map_y, p)
+                       : cudaLaunchKernelEx(&cfg, gemm_i8_kernel<kSparse, GPUSQ_OUT_I32>, map_a, map_b, map_e, map_y, p);
     if (err != cudaSuccess) {
         (void)cudaGetLastError();
         return GPUSQ_ERR_CUDA;
@@ -1093,11 +1122,12 @@ static int launch_gemm_f16(const void *X, const void *Wpacked, const float *bias
     static std::once_flag attr_once;
     static cudaError_t attr_err = cudaSuccess;
     std::call_once(attr_once, [] {
-        attr_err = cudaFuncSetAttribute(gemm_i8_kernel<true, GPUSQ_OUT_F16, true>,
-                                        cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
-        if (attr_err == cudaSuccess)
-            attr_err = cudaFuncSetAttribute(gemm_i8_kernel<true, GPUSQ_OUT_I32, true>,
-                                            cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+        const void *kernels[4] = {
+            (const void *)gemm_i8_kernel<true, GPUSQ_OUT_F16, true>, (const void *)gemm_i8_kernel<true, GPUSQ_OUT_I32, true>,
+            (const void *)gemm_i8_kernel<true, GPUSQ_OUT_F16, true, true>,
+            (const void *)gemm_i8_kernel<true, GPUSQ_OUT_I32, true, true>};
+        for (int k = 0; k < 4 && attr_err == cudaSuccess; ++k)
+            attr_err = cudaFuncSetAttribute(kernels[k], cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
     });
     if (attr_err != cudaSuccess) return GPUSQ_ERR_CUDA;
 
@@ -1105,9 +1135,10 @@ static int launch_gemm_f16(const void *X, const void *Wpacked, const float *bias
     const int clusters = max_clusters<true, true>(sms);
     if (clusters <= 0) return GPUSQ_ERR_CUDA;
     const int tiles_n = (N + kPairF - 1) / kPairF;
-    const bool twin = N <= kBlockF && M < 0x7FFFFFFF - 4 * kMaxBlockT;
+    const bool twin_col = N - (tiles_n - 1) * kPairF <= kBlockF && M < 0x7FFFFFFF - 4 * kMaxBlockT;
     // twice the bytes per column
-    const int block_t = twin ? choose_block_t(ceil_div(M, 2), 1, clusters, 4 * K) : choose_block_t(M, tiles_n, clusters, 2 * K);
+    const int block_t = (twin_col && tiles_n == 1) ? choose_block_t(ceil_div(M, 2), 1, clusters, 4 * K)
+                                                   : choose_block_t(M, tiles_n, clusters, 2 * K);
     const int Kp = round_up(K, 128), Np = round_up(N, kPairF);
 
     // every tensor is described in bytes: kept values [Np, Kp] (Kp / 2 binary16 per row), activations
@@ -1136,10 +1167,15 @@ static int launch_gemm_f16(const void *X, const void *Wpacked, const float *bias
     p.block_t = block_t;
     p.act = act;
     p.out_type = out_type;
-    p.twin = twin ? 1 : 0;
+    p.pair_cols = twin_col ? tiles_n - 1 : tiles_n;
+    const int64_t pair_tiles = (int64_t)p.pair_cols * ceil_div(M, block_t);
+    const int64_t tiles = pair_tiles + (twin_col ? ceil_div(M, 2 * (int64_t)block_t) : 0);
+    if (tiles > 0x7FFFFFFF) return GPUSQ_ERR_SHAPE;
+    p.pair_tiles = (int)pair_tiles;
+    p.num_tiles = (int)tiles;
+    p.twin_n0 = p.pair_cols * kPairF;
     p.oob_row = Np;
 
-    const int64_t tiles = twin ? ceil_div(M, 2 * (int64_t)block_t) : (int64_t)tiles_n * ceil_div(M, block_t);
     const int grid = 2 * (int)(tiles < clusters ? tiles : clusters);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid, 1, 1);
@@ -1153,9 +1189,11 @@ static int launch_gemm_f16(const void *X, const void *Wpacked, const float *bias
     cfg.numAttrs = 1;
     cudaError_t err;
     if (out_type == GPUSQ_OUT_F16)
-        err = cudaLaunchKernelEx(&cfg, gemm_i8_kernel<true, GPUSQ_OUT_F16, true>, map_a, map_b, map_e, map_y, p);
+        err = twin_col ? cudaLaunchKernelEx(&cfg, gemm_i8_kernel<true, GPUSQ_OUT_F16, true, true>, map_a, map_b, map_e, map_y, p)
+                       : cudaLaunchKernelEx(&cfg, gemm_i8_kernel<true, GPUSQ_OUT_F16, true>, map_a, map_b, map_e, map_y, p);
     else
-        err = cudaLaunchKernelEx(&cfg, gemm_i8_kernel<true, GPUSQ_OUT_I32, true>, map_a, map_b, map_e, map_y, p);
+        err = twin_col ? cudaLaunchKernelEx(&cfg, gemm_i8_kernel<true, GPUSQ_OUT_I32, true, true>, map_a, map_b, map_e, map_y, p)
+                       : cudaLaunchKernelEx(&cfg, gemm_i8_kernel<true, GPUSQ_OUT_I32, true>, map_a, map_b, map_e, map_y, p);
     if (err != cudaSuccess) {
         (void)cudaGetLastError();
         return GPUSQ_ERR_CUDA;
