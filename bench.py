@@ -40,7 +40,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum of the four sparse-GEMM launches of one step, from the
 # ncu capture summarised in profiles/gemm_i8_sparse_deit_base_block.md (cold L2 per launch: most of
 # the FP16 output is still in L2 when a launch ends).  Set to None when the kernel changes.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 96.0e6
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 94.4e6
 
 
 def load_peaks():
