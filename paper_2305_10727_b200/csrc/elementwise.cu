@@ -798,7 +798,9 @@ int gpusq_quant_act(const void *X, int8_t *Xq, float *x_scale, int scale_mode, i
             return GPUSQ_ERR_CUDA;
         int grid = num_sms();
         if (grid > kMaxPartials) grid = kMaxPartials;
-        if ((int64_t)grid > vec8) grid = (int)vec8;
+        // small tensors: no more CTAs than give every thread two vectors (fewer arrivals at the barrier)
+        const int64_t want = ceil_div(vec8, 2 * kFusedThreads);
+        if ((int64_t)grid > want) grid = (int)(want < 1 ? 1 : want);
         if (ceil_div(vec8, grid) > 0x7FFFFFFF) return GPUSQ_ERR_SHAPE;      // a CTA's slice is indexed with 32 bits
         uint32_t *counters = reinterpret_cast<uint32_t *>(workspace) + kMaxPartials;
         const uint4 *Xv = reinterpret_cast<const uint4 *>(X);
