@@ -1,6 +1,7 @@
 /*
  * gpusq -- 2:4 fine-grained structured-sparse INT8 linear layers for NVIDIA
- * B200 (sm_100a).  C ABI of libgpusq.so.
+ * B200 (sm_100a), the patch-embedding layer on the same GEMM, and the FP16 2:4
+ * sparse model the INT8 one is quantised from.  C ABI of libgpusq.so.
  *
  * The layer is Y = X * W^T with
  *   W [N, K]  weight: the 2:4-sparse operand (matrix A of the paper's Fig. 1)
@@ -43,7 +44,7 @@ typedef enum gpusq_status {
     GPUSQ_ERR_CUDA = 6,             /* a CUDA runtime / driver call failed */
     GPUSQ_ERR_TIMEOUT = 7,          /* a bounded device-side wait expired (see status_buf) */
     GPUSQ_ERR_ARG = 8,              /* an enum argument is out of range */
-    GPUSQ_ERR_TOO_LARGE = 9         /* the tensor exceeds the fixed capacity of a *_static entry point */
+    GPUSQ_ERR_TOO_LARGE = 9         /* the tensor exceeds the fixed capacity of the entry point */
 } gpusq_status;
 
 enum { GPUSQ_ACT_NONE = 0, GPUSQ_ACT_GELU = 1 };
