@@ -7,6 +7,7 @@ or imports the product package.
 """
 from .oracle import (  # noqa: F401
     build,
+    host_cores,
     prune24,
     quant_weight,
     compress24,

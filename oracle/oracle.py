@@ -9,6 +9,7 @@ import ctypes
 import os
 import subprocess
 import threading
+from concurrent.futures import ThreadPoolExecutor
 
 import numpy as np
 
@@ -88,6 +89,34 @@ def _c(a, dtype):
     return a
 
 
+def host_cores() -> int:
+    """Cores this process may run on."""
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+def _row_blocks(n_rows: int, threads: int):
+    """Contiguous row ranges, a few per thread so that uneven speeds even out."""
+    parts = max(1, min(n_rows, 4 * threads))
+    edges = [n_rows * i // parts for i in range(parts + 1)]
+    return [(a, b) for a, b in zip(edges[:-1], edges[1:]) if b > a]
+
+
+def _over_row_blocks(n_rows: int, threads, fn):
+    """Run fn(lo, hi) over row blocks: output rows are independent of one another, so the plain
+    single-threaded C routine is simply called once per block, from several Python threads when
+    threads > 1 (ctypes releases the interpreter lock during the call).  The arithmetic is the C
+    file's in either case; only which call computes which rows differs."""
+    if not threads or threads <= 1 or n_rows < 2:
+        fn(0, n_rows)
+        return
+    with ThreadPoolExecutor(max_workers=threads) as pool:
+        for f in [pool.submit(fn, lo, hi) for lo, hi in _row_blocks(n_rows, threads)]:
+            f.result()
+
+
 def prune24(W, return_mask=False):
     W = _c(W, np.float32)
     N, K = W.shape
@@ -141,14 +170,21 @@ def quant_act(X, x_scale=None):
     return Xq, np.float32(s[0])
 
 
-def spgemm_acc(Xq, vals, meta):
+def spgemm_acc(Xq, vals, meta, threads=None):
+    """threads > 1: the token rows are split into blocks, one plain o_spgemm_acc call per block."""
     Xq, vals, meta = _c(Xq, np.int8), _c(vals, np.int8), _c(meta, np.uint8)
     M, K = Xq.shape
     N = vals.shape[0]
     assert vals.shape == (N, K // 2) and meta.shape == (N, K // 8)
     acc = np.empty((M, N), np.int32)
-    ovf = _load().o_spgemm_acc(_p(Xq), _p(vals), _p(meta), _p(acc), M, N, K)
-    assert ovf == 0, "INT32 overflow in %d sums" % ovf
+    lib = _load()
+    overflow = []
+
+    def block(lo, hi):
+        overflow.append(lib.o_spgemm_acc(_p(Xq[lo:hi]), _p(vals), _p(meta), _p(acc[lo:hi]), hi - lo, N, K))
+
+    _over_row_blocks(M, threads, block)
+    assert sum(overflow) == 0, "INT32 overflow in %d sums" % sum(overflow)
     return acc
 
 
@@ -192,15 +228,22 @@ def patch_conv_acc(imgq, Wq4):
 _OUT_DTYPES = {0: np.float16, 1: np.int8, 2: np.int32}
 
 
-def epilogue(acc, w_scale, x_scale, bias=None, act=0, out_type=0, out_scale=1.0):
+def epilogue(acc, w_scale, x_scale, bias=None, act=0, out_type=0, out_scale=1.0, threads=None):
+    """threads > 1: one plain o_epilogue call per block of whole rows."""
     acc = _c(acc, np.int32)
     w_scale = _c(w_scale, np.float32)
     if bias is not None:
         bias = _c(bias, np.float32)
     N = acc.shape[-1]
     Y = np.empty(acc.shape, _OUT_DTYPES[out_type])
-    _load().o_epilogue(_p(acc), _p(w_scale), float(x_scale), _p(bias), act, out_type,
-                       float(out_scale), _p(Y), acc.size, N)
+    lib = _load()
+    acc2, Y2 = acc.reshape(-1, N), Y.reshape(-1, N)
+
+    def block(lo, hi):
+        lib.o_epilogue(_p(acc2[lo:hi]), _p(w_scale), float(x_scale), _p(bias), act, out_type,
+                       float(out_scale), _p(Y2[lo:hi]), (hi - lo) * N, N)
+
+    _over_row_blocks(acc2.shape[0], threads, block)
     return Y
 
 
@@ -228,17 +271,19 @@ def prepare_weight(W):
 
 
 def layer_forward(X, prep, bias=None, act=0, out_type=0, out_scale=1.0, x_scale=None,
-                  rows=None):
+                  rows=None, threads=None):
     """Per-inference call: quantise activations -> sparse GEMM -> epilogue.
 
     rows: optional token-row subset (the activation scale still comes from all of X).
+    threads: GEMM and epilogue over row blocks on that many host threads (see _over_row_blocks);
+    the activation quantisation, whose scale needs the whole tensor, stays one call.
     """
     Xq, xs = quant_act(X, x_scale)
     if rows is None:
-        acc = spgemm_acc(Xq, prep["vals"], prep["meta"])
+        acc = spgemm_acc(Xq, prep["vals"], prep["meta"], threads=threads)
     else:
         acc = spgemm_acc_rows(Xq, prep["vals"], prep["meta"], rows)
-    Y = epilogue(acc, prep["w_scale"], xs, bias, act, out_type, out_scale)
+    Y = epilogue(acc, prep["w_scale"], xs, bias, act, out_type, out_scale, threads=threads)
     return {"Xq": Xq, "x_scale": xs, "acc": acc, "Y": Y}
 
 

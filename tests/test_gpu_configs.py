@@ -1,10 +1,15 @@
 """GPU parity at the full benchmark sizes, in the launch configuration bench.py
 times (automatic tile choice, persistent grid): every workload config,
 every layer.  Weight-side stages and the activation codes are compared with the
-oracle in full; the GEMM and the epilogue are compared on sampled token rows the
-oracle computes one by one (first tile, the ragged last tile, random rows), plus
-an exact column-sum identity that covers every output element, plus equality
-with the dense-instruction variant of the same kernel."""
+oracle in full.  For the config the benchmark is quoted on (DeiT-Base block,
+batch 64) the INT32 accumulators and the FP16 output of ALL token rows of every
+layer are compared with the oracle element by element (the plain oracle, its
+row blocks spread over the host's cores).  For the other configs, whose GEMMs
+would take the oracle minutes to hours, the GEMM and the epilogue are compared
+on sampled token rows the oracle computes one by one (first tile, the ragged
+last tile, random rows), plus an exact column-sum identity that covers every
+output element, plus equality with the dense-instruction variant of the same
+kernel."""
 import numpy as np
 import pytest
 
@@ -15,6 +20,7 @@ torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
 
 F16_ULP_TOL = 1
+FULL_COMPARE = ("deit_base_b64", "deit_tiny_fc1", "deit_tiny_b64")     # every output element against the oracle
 
 
 @pytest.fixture(scope="module")
@@ -79,8 +85,12 @@ def test_config_layer(B, name, li):
     acc_dense = B.gemm_i8_dense(Xq, Wq, out_type=B.OUT_I32, status_buf=status)
     assert status.cpu().tolist() == [0, 0, 0, 0]
     assert torch.equal(acc, acc_dense)                   # same C as the dense GEMM, every element
-    rows = sample_rows(M, cfg.cid * 10 + li)
-    acc_rows_o = oracle.spgemm_acc_rows(Xq_o, prep["vals"], prep["meta"], rows)
+    if name in FULL_COMPARE:
+        rows = np.arange(M, dtype=np.int64)
+        acc_rows_o = oracle.spgemm_acc(Xq_o, prep["vals"], prep["meta"], threads=oracle.host_cores())
+    else:
+        rows = sample_rows(M, cfg.cid * 10 + li)
+        acc_rows_o = oracle.spgemm_acc_rows(Xq_o, prep["vals"], prep["meta"], rows)
     assert np.array_equal(acc[cu(rows)].cpu().numpy(), acc_rows_o)
     # sum_m acc[m, n] = sum_k Wq[n, k] * (sum_m Xq[m, k]): exact in int64, touches every element
     col = acc.sum(dim=0, dtype=torch.int64).cpu().numpy()
@@ -92,7 +102,8 @@ def test_config_layer(B, name, li):
     act = 1 if L.gelu else 0
     bias = cu(d["bias"])
     Y = B.spgemm_i8(Xq, Wpk, L.N, ws, xs, bias, act=act, out_type=B.OUT_F16, status_buf=status)
-    Y_rows_o = oracle.epilogue(acc_rows_o, prep["w_scale"], xs_o, d["bias"], act=act, out_type=0)
+    Y_rows_o = oracle.epilogue(acc_rows_o, prep["w_scale"], xs_o, d["bias"], act=act, out_type=0,
+                               threads=oracle.host_cores())
     dist = f16_ulp_distance(Y[cu(rows)].cpu().numpy(), Y_rows_o)
     assert dist.max() <= F16_ULP_TOL
     if act == 0:
@@ -105,7 +116,8 @@ def test_config_layer(B, name, li):
         Q = B.spgemm_i8(Xq, Wpk, L.N, ws, xs, bias, act=act, out_type=B.OUT_I8,
                         out_scale=cu(np.array([out_scale], np.float32)), status_buf=status)
         Q_rows_o = oracle.epilogue(acc_rows_o, prep["w_scale"], xs_o, d["bias"], act=act, out_type=1,
-                                   out_scale=out_scale)
+                                   out_scale=out_scale, threads=oracle.host_cores())
         diff = np.abs(Q[cu(rows)].cpu().numpy().astype(np.int32) - Q_rows_o.astype(np.int32))
         assert diff.max() <= (1 if act else 0)
+        assert (diff != 0).sum() <= max(1, int(1e-3 * diff.size))
     assert status.cpu().tolist() == [0, 0, 0, 0]

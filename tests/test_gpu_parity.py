@@ -355,3 +355,6 @@ def test_layer_random_shapes(B, i, M, N, K, block_t, act, use_bias):
     if Q is not None:
         diff = np.abs(Q.astype(np.int32) - Q_o.astype(np.int32))
         assert diff.max() <= (1 if act else 0)
+        # with GELU a code may flip only at a rounding tie: fewer than one in a thousand (at least
+        # one element is always allowed, so that tiny outputs are not held to a stricter bar)
+        assert (diff != 0).sum() <= max(1, int(1e-3 * diff.size))

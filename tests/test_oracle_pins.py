@@ -323,6 +323,33 @@ def test_layer_forward_composition_and_sqnr():
     assert np.array_equal(sub["Y"], out["Y"][rows])
 
 
+def test_sqnr_hand_value():
+    # ref = [1, 1], test = [1, 0.9]: signal 2, noise 0.01 -> 10 log10(200) dB; equal scaling of both leaves it alone
+    want = 10.0 * np.log10(200.0)
+    got = oracle.sqnr_db(np.array([1.0, 1.0], np.float32), np.array([1.0, 0.9], np.float32))
+    assert abs(got - want) < 1e-5                        # 0.9 is not exact in binary32
+    assert abs(oracle.sqnr_db(np.array([4.0, 4.0], np.float32), np.array([4.0, 3.5], np.float32))
+               - 10.0 * np.log10(32.0 / 0.25)) < 1e-12   # exact inputs: 21.07 dB
+
+
+def test_row_parallel_driver_equals_single_thread():
+    # the several-thread driver only splits the token rows over plain calls of the same C routines:
+    # on the whole of the small workload config its results equal the single-threaded ones bit for bit
+    cfg = inputs.CONFIGS["deit_tiny_fc1"]
+    d = inputs.make_layer_inputs(cfg, 0)
+    prep = oracle.prepare_weight(d["W"])
+    one = oracle.layer_forward(d["X"], prep, d["bias"], act=1)
+    for threads in (2, 3, 7):
+        many = oracle.layer_forward(d["X"], prep, d["bias"], act=1, threads=threads)
+        assert np.array_equal(one["acc"], many["acc"])
+        assert np.array_equal(one["Y"].view(np.uint16), many["Y"].view(np.uint16))
+    q1 = oracle.epilogue(one["acc"], prep["w_scale"], one["x_scale"], d["bias"], act=1, out_type=1, out_scale=0.01)
+    q4 = oracle.epilogue(one["acc"], prep["w_scale"], one["x_scale"], d["bias"], act=1, out_type=1, out_scale=0.01,
+                         threads=4)
+    assert np.array_equal(q1, q4)
+    assert oracle.host_cores() >= 1
+
+
 # ---------------------------------------------------------------- patch embedding (Sec. 3.3)
 
 PATCH_SHAPES = [(2, 3, 8, 8, 4, 5), (1, 3, 28, 42, 14, 7), (3, 2, 32, 16, 16, 4), (2, 1, 6, 4, 2, 3)]

@@ -5,9 +5,9 @@ quantised (memory planned and frozen by a serving framework, allocator calls
 banned in a latency-critical loop, a fixed budget owned by someone else), so
 this entry point works out of a fixed array inside the library.  The test calls
 it through the C ABI twice in a row and checks both results, bit for bit,
-against the ordinary entry point -- the second call on a smaller tensor with a
-smaller maximum, so anything left in the shared scratch by the first call would
-show up as a wrong scale.  This file sorts last on purpose: a run that stops at
+against the ordinary entry point and against the CPU oracle -- the second call
+on a smaller tensor with a smaller maximum, so anything left in the shared
+scratch by the first call would show up as a wrong scale.  This file sorts last on purpose: a run that stops at
 the first failure has then already run every other test.
 """
 import ctypes
@@ -15,6 +15,7 @@ import ctypes
 import numpy as np
 import pytest
 
+import oracle
 from paper_2305_10727_b200 import inputs
 
 torch = pytest.importorskip("torch")
@@ -42,6 +43,9 @@ def test_static_entry_point_matches_workspace_entry_point_twice():
         torch.cuda.synchronize()
         assert s.item() == s_ref.item()                                   # integer stage: bit-exact
         assert torch.equal(Xq, Xq_ref)
+        Xq_o, s_o = oracle.quant_act(X_host)                              # the definition, on the CPU
+        assert s.cpu().numpy()[0] == s_o
+        assert np.array_equal(Xq.cpu().numpy(), Xq_o)
 
     # a supplied scale goes through the same entry point without touching the scratch
     X = torch.from_numpy(big).cuda()
@@ -49,6 +53,7 @@ def test_static_entry_point_matches_workspace_entry_point_twice():
     Xq_ref, _ = B.quant_act(X, x_scale=given, scale_mode=B.SCALE_GIVEN)
     Xq, _ = B.quant_act_static(X, x_scale=given, scale_mode=B.SCALE_GIVEN)
     assert torch.equal(Xq, Xq_ref)
+    assert np.array_equal(Xq.cpu().numpy(), oracle.quant_act(big, x_scale=np.float32(0.02))[0])
 
     # beyond the stated capacity: refused, nothing enqueued
     rc = lib.gpusq_quant_act_static(ctypes.c_void_p(X.data_ptr()), ctypes.c_void_p(Xq.data_ptr()),
