@@ -34,13 +34,38 @@ from paper_2305_10727_b200 import inputs  # noqa: E402
 
 METRIC = "sparse INT8 GEMM effective TOPS (dense-equivalent 2*M*N*K / time), ViT-B block linears at batch 64"
 UNIT = "TOPS"
+STEP_TEXT = "per layer: quant_act (per-tensor absmax scale + quantise) + sparse GEMM with fused epilogue, FP16 out"
 NOMINAL_SPARSE_INT8_TOPS = 9000.0      # NVIDIA's dense-half figure for B200 INT8 with 2:4 sparsity (4 x 2250 BF16)
 NOMINAL_BF16_TFLOPS = 2250.0
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# dram__bytes_read.sum + dram__bytes_write.sum of the four sparse-GEMM launches of one step, from the
-# ncu capture summarised in profiles/gemm_i8_sparse_deit_base_block.md (cold L2 per launch: most of
-# the FP16 output is still in L2 when a launch ends).  Set to None when the kernel changes.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 94.4e6
+# DRAM traffic of the step's GEMM launches comes from the ncu summary committed under profiles/ (a line
+# "dram_bytes_gemm_launches_per_step <bytes> kernel_sha <sha>"); it is reported only while the kernel
+# sources still hash to the value recorded there.
+TRAFFIC_SUMMARY = os.path.join(ROOT, "profiles", "gemm_i8_sparse_deit_base_block.md")
+KERNEL_SOURCES = ("gemm_i8.cu", "ptx.cuh", "quant_math.cuh", "common.cuh")
+
+
+def kernel_sha():
+    import hashlib
+    h = hashlib.sha256()
+    for name in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, "paper_2305_10727_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def recorded_traffic(workload_key):
+    """(bytes per step, launches) of the GEMM launches from the committed ncu summary, or (None, None)."""
+    try:
+        with open(TRAFFIC_SUMMARY) as f:
+            for line in f:
+                parts = line.split()
+                if len(parts) >= 7 and parts[0] == "dram_bytes_gemm_launches_per_step" and parts[1] == workload_key:
+                    if parts[6] == kernel_sha():
+                        return float(parts[2]), int(parts[4])
+    except OSError:
+        pass
+    return None, None
 
 
 def load_peaks():
@@ -140,9 +165,11 @@ def run_reference(args, cfg):
             data.append((L, d, oracle.prepare_weight(d["W"])))
         return data
 
+    cores = oracle.host_cores()
+
     def step(data):
         for L, d, prep in data:
-            oracle.layer_forward(d["X"], prep, d["bias"], act=1 if L.gelu else 0)
+            oracle.layer_forward(d["X"], prep, d["bias"], act=1 if L.gelu else 0, threads=cores)
 
     rows = args.ref_rows
     if rows <= 0:
@@ -152,7 +179,7 @@ def run_reference(args, cfg):
         per_row = (time.perf_counter() - t0) / 16
         budget_s = 60.0
         rows = int(budget_s / max(per_row, 1e-9) / (args.steps + args.warmup))
-        rows = max(4, min(rows, 512, cfg.M))
+        rows = max(4 * cores, min(rows, 512 * cores, cfg.M))
     data = make(rows)
     flops = sum(layer_flops(rows, L) for L in layers)
     for _ in range(args.warmup):
@@ -168,8 +195,10 @@ def run_reference(args, cfg):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3 * (cfg.M / rows),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
         "config": {"workload": cfg.name, "M": cfg.M, "layers": [[L.name, L.K, L.N] for L in layers],
+                   "step": STEP_TEXT, "launch": "host threads", "l2": "not applicable (CPU)",
+                   "parallelism": "%d host threads over row blocks" % cores,
                    "note": "ms_per_step is the sampled step scaled to all M rows"},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -326,13 +355,19 @@ def run_gpusq(args, cfg):
         return fn
 
     all_idx = tuple(range(len(state)))
+    single = len(state) == 1            # a one-layer step: leaving the layer out leaves nothing to time
     ms_full = loop_ms(step_without())
     ms_no_gemm = loop_ms(step_without(skip_gemm=all_idx))
+    ms_no_quant = loop_ms(step_without(skip_quant=all_idx))
     gemm_us, quant_us, dense_us = {}, {}, {}
     for i, s in enumerate(state):
         name = s["L"].name
-        gemm_us[name] = [max(ms_full - loop_ms(step_without(skip_gemm=(i,))), 1e-3) * 1e3]
-        quant_us[name] = [max(ms_full - loop_ms(step_without(skip_quant=(i,))), 1e-3) * 1e3]
+        if single:
+            gemm_us[name] = [max(ms_full - ms_no_gemm, 1e-3) * 1e3]
+            quant_us[name] = [max(ms_full - ms_no_quant, 1e-3) * 1e3]
+        else:
+            gemm_us[name] = [max(ms_full - loop_ms(step_without(skip_gemm=(i,))), 1e-3) * 1e3]
+            quant_us[name] = [max(ms_full - loop_ms(step_without(skip_quant=(i,))), 1e-3) * 1e3]
     # the same step with the activation scales supplied (calibrated once, as the paper's deployed model
     # does with its learned scales) instead of computed from every batch: extra information
     def step_static_scale():
@@ -390,11 +425,13 @@ def run_gpusq(args, cfg):
             return fn
         ms_half = loop_ms(step_half())
         for i, s in enumerate(state):
-            half_layer_us[s["L"].name] = round(max(ms_half - loop_ms(step_half(skip=(i,))), 1e-3) * 1e3, 2)
+            half_layer_us[s["L"].name] = round((ms_half if single else
+                                                max(ms_half - loop_ms(step_half(skip=(i,))), 1e-3)) * 1e3, 2)
     ms_dense = loop_ms(step_without(gemm=layer_gemm_dense))
     for i, s in enumerate(state):
         name = s["L"].name
-        dense_us[name] = [max(ms_dense - loop_ms(step_without(skip_gemm=(i,), gemm=layer_gemm_dense)), 1e-3) * 1e3]
+        dense_us[name] = [max(ms_dense - (ms_no_gemm if single else
+                                          loop_ms(step_without(skip_gemm=(i,), gemm=layer_gemm_dense))), 1e-3) * 1e3]
     gemm_block_us = (ms_full - ms_no_gemm) * 1e3
     dense_block_us = (ms_dense - ms_no_gemm) * 1e3
     clocks = sampler.stop()
@@ -405,14 +442,23 @@ def run_gpusq(args, cfg):
     flops_step = sum(layer_flops(M, L) for L in layers)
     value = replicas.whole_job_throughput(flops_step, ms_step * 1e-3, world) / 1e12
 
-    # ---- roofline of the dominant kernel (the sparse GEMM, all four shapes of the block)
+    # ---- roofline of the dominant kernel (the sparse GEMM, all shapes of the step).  Two roofs: the tensor
+    # pipe (dense-equivalent ops / peak) and HBM (algorithmic bytes / measured copy bandwidth); the one
+    # that needs the longer time for these shapes binds, and `frac` is the fraction of THAT roof.  The
+    # tensor peak is derived from the measured cuBLAS BF16 figure of the regime the timed region ran in
+    # (burst: milliseconds at full clocks; sustained: a seconds-long loop under the power cap) times the
+    # nominal INT8-2:4 : BF16 ratio; the fraction of the nominal 9000 TOPS is reported beside it.
     gemm_mean = {k: statistics.fmean(v) for k, v in gemm_us.items()}
     gemm_total_us = gemm_block_us
     achieved = flops_step / (gemm_total_us * 1e-6) / 1e12
     sparse_ratio = NOMINAL_SPARSE_INT8_TOPS / NOMINAL_BF16_TFLOPS
-    peak = peaks["bf16_tflops_sustained"] * sparse_ratio
+    timed_region_s = ms_step * 1e-3 * args.steps
+    regime = "burst" if timed_region_s < 1.0 else "sustained"
+    tensor_peak = (peaks["bf16_tflops"] if regime == "burst" else peaks["bf16_tflops_sustained"]) * sparse_ratio
     bytes_step = sum(layer_bytes(M, L) for L in layers)
     hbm_achieved = bytes_step / (gemm_total_us * 1e-6) / 1e9
+    t_tensor_us = flops_step / (tensor_peak * 1e12) * 1e6
+    t_hbm_us = bytes_step / (peaks["hbm_gbs"] * 1e9) * 1e6
     per_layer = {}
     for L in layers:
         us = gemm_mean[L.name]
@@ -421,23 +467,36 @@ def run_gpusq(args, cfg):
             "tops": round(layer_flops(M, L) / us / 1e6, 1),
             "frac_nominal_sparse_peak": round(layer_flops(M, L) / us / 1e6 / NOMINAL_SPARSE_INT8_TOPS, 4),
             "hbm_gbs": round(layer_bytes(M, L) / us / 1e3, 1),
+            "hbm_frac": round(layer_bytes(M, L) / us / 1e3 / peaks["hbm_gbs"], 4),
             "dense_variant_us": round(statistics.fmean(dense_us[L.name]), 2),
             "speedup_vs_dense_variant": round(statistics.fmean(dense_us[L.name]) / us, 3),
             "quant_act_us": round(statistics.fmean(quant_us[L.name]), 2),
         }
-    roofline = {
-        "bound": "tensor", "kernel": "gemm_i8_kernel<sparse>", "achieved": round(achieved, 1),
-        "peak": round(peak, 1), "unit": "TFLOP/s", "frac": round(achieved / peak, 4),
-        "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH if args.config == "deit_base_b64" else None,
-        "peak_source": "%s BF16 sustained x %.0f (nominal INT8-sparse : BF16 ratio)" % (peaks["_source"], sparse_ratio),
+    traffic, traffic_launches = recorded_traffic(args.config)
+    common = {
+        "kernel": "gemm_i8_kernel<sparse>", "launches_per_step": len(layers),
+        "traffic": traffic, "traffic_note": None if traffic is None else
+        "ncu dram__bytes_read.sum + dram__bytes_write.sum summed over the %d GEMM launches of one step, L2 not flushed "
+        "between launches (profiles/gemm_i8_sparse_deit_base_block.md)" % traffic_launches,
+        "algorithmic_bytes": bytes_step, "tensor_time_us": round(t_tensor_us, 2), "hbm_time_us": round(t_hbm_us, 2),
+        "tensor_achieved_tops": round(achieved, 1), "tensor_peak_tops": round(tensor_peak, 1),
+        "tensor_peak_source": "%s BF16 %s x %.0f (nominal INT8-sparse : BF16 ratio)" % (peaks["_source"], regime, sparse_ratio),
+        "tensor_frac": round(achieved / tensor_peak, 4),
         "frac_of_nominal_9000": round(achieved / NOMINAL_SPARSE_INT8_TOPS, 4),
-        "frac_of_burst_peak": round(achieved / (peaks["bf16_tflops"] * sparse_ratio), 4),
         "hbm_achieved_gbs": round(hbm_achieved, 1), "hbm_peak_gbs": peaks["hbm_gbs"],
         "hbm_frac": round(hbm_achieved / peaks["hbm_gbs"], 4),
         "gemm_block_us": round(gemm_total_us, 2),
         "timing": "CUDA events around %d replays of the step with and without the GEMM launches; the difference is the GEMMs' time in context" % args.steps,
         "dense_variant_block_us": round(dense_block_us, 2), "speedup_vs_dense_variant": round(dense_block_us / gemm_block_us, 3),
     }
+    if t_hbm_us >= t_tensor_us:
+        roofline = {"bound": "hbm", "achieved": round(hbm_achieved, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": round(hbm_achieved / peaks["hbm_gbs"], 4),
+                    "peak_source": "%s copy bandwidth" % peaks["_source"]}
+    else:
+        roofline = {"bound": "tensor", "achieved": round(achieved, 1), "peak": round(tensor_peak, 1), "unit": "TFLOP/s",
+                    "frac": round(achieved / tensor_peak, 4), "peak_source": common["tensor_peak_source"]}
+    roofline.update(common)
 
     # ---- end to end through the public API with host buffers (pinned), copies inside the timed region
     e2e = None
@@ -494,23 +553,32 @@ def run_gpusq(args, cfg):
         e2e = {"value": round(world * flops_step / (ms_e2e * 1e-3) / 1e12, 2), "unit": UNIT,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": round(ms_e2e, 4), "steps": n_e2e}
 
-    # ---- CPU baseline: the oracle on a bounded sample (rank 0, N = 1 only)
+    # ---- CPU baseline: the oracle on a bounded sample (rank 0, N = 1 only): on one core, and with its
+    # row blocks spread over all host cores (the same plain routines, called once per block of rows)
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle
-        rows = args.ref_rows
-        t_cpu = 0.0
-        for li, L in enumerate(layers):
-            h = host[li]
-            prep = oracle.prepare_weight(h["W"])
-            Xs = np.ascontiguousarray(h["X"][:rows])
-            t0 = time.perf_counter()
-            oracle.layer_forward(Xs, prep, h["bias"], act=1 if L.gelu else 0)
-            t_cpu += time.perf_counter() - t0
-        cpu_tops = sum(layer_flops(rows, L) for L in layers) / t_cpu / 1e12
-        cpu_baseline = {"value": cpu_tops, "unit": UNIT, "cores": 1, "kind": "oracle",
-                        "sample": "first %d of %d token rows of each layer (quantise + GEMM + epilogue), %.1f s"
-                                  % (rows, M, t_cpu)}
+        cores = oracle.host_cores()
+        rows_all = min(M, args.ref_rows)
+        rows_one = min(M, max(256, args.ref_rows // 4))
+        preps = [oracle.prepare_weight(host[li]["W"]) for li in range(len(layers))]
+
+        def oracle_seconds(rows, threads):
+            t = 0.0
+            for li, L in enumerate(layers):
+                Xs = np.ascontiguousarray(host[li]["X"][:rows])
+                t0 = time.perf_counter()
+                oracle.layer_forward(Xs, preps[li], host[li]["bias"], act=1 if L.gelu else 0, threads=threads)
+                t += time.perf_counter() - t0
+            return t
+
+        t_one = oracle_seconds(rows_one, 1)
+        t_all = oracle_seconds(rows_all, cores)
+        tops_one = sum(layer_flops(rows_one, L) for L in layers) / t_one / 1e12
+        tops_all = sum(layer_flops(rows_all, L) for L in layers) / t_all / 1e12
+        cpu_baseline = {"value": tops_all, "unit": UNIT, "cores": cores, "kind": "oracle", "value_1core": tops_one,
+                        "sample": "quantise + GEMM + epilogue of every layer: first %d of %d token rows on %d cores (%.1f s), "
+                                  "first %d rows on one core (%.1f s)" % (rows_all, M, cores, t_all, rows_one, t_one)}
 
     if rank == 0:
         line = {
@@ -518,11 +586,12 @@ def run_gpusq(args, cfg):
             "warmup": max(args.warmup, 3), "ms_per_step": round(ms_step, 5), "block_us": round(ms_step * 1e3, 2),
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
             "config": {"workload": cfg.name, "M": M, "layers": [[L.name, L.K, L.N] for L in layers],
-                       "step": "per layer: quant_act (per-tensor absmax scale + quantise, one launch) + sparse GEMM with fused epilogue, FP16 out",
+                       "step": STEP_TEXT,
                        "launch": args.launch, "l2": "inputs exceed L2: a step touches %.0f MB" % ((bytes_step + sum(2.0 * M * L.K for L in layers)) / 1e6),
                        "parallelism": "replicas, tokens sharded, no collective" if world > 1 else "single GPU"},
             "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e,
             "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
+            "step_us_x_sm_mhz": None if not clocks.get("sm_mhz") else round(ms_step * 1e3 * clocks["sm_mhz"], 1),
             "layers": per_layer, "prep_us": {k: round(v, 2) for k, v in prep_us.items()},
             "static_scale_step": {"block_us": round(ms_static * 1e3, 2),
                                   "value": round(flops_step / (ms_static * 1e-3) / 1e12, 2), "unit": UNIT,
@@ -702,8 +771,8 @@ def main():
     ap.add_argument("--patch", default=None, choices=list(inputs.PATCH_CONFIGS),
                     help="measure a patch-embedding workload instead of a block of linear layers")
     ap.add_argument("--launch", default="graph", choices=["graph", "eager"])
-    ap.add_argument("--ref-rows", type=int, default=4096,
-                    help="token rows per layer the CPU oracle is timed on (about 15 s of single-core work)")
+    ap.add_argument("--ref-rows", type=int, default=8192,
+                    help="token rows per layer the CPU oracle is timed on with all host cores (a quarter of them on one core)")
     ap.add_argument("--ref-rows-reference", type=int, default=0,
                     help="token rows per step for --impl reference (0 = size from a calibration run)")
     ap.add_argument("--no-e2e", action="store_true")
