@@ -264,14 +264,6 @@ int gpusq_gemm_i8_dense(const int8_t *Xq, const int8_t *Wq, const float *w_scale
                         const float *out_scale, void *Y, int64_t M, int N, int K,
                         int32_t *status_buf, void *stream);
 
-/* ---------------------------------------------------------------------------
- * gpusq_set_block_tokens -- tuning hook for the two GEMM calls (the paper has
- * no counterpart).  block_t = tokens per output tile, a multiple of 32 in
- * [32, 224]; 0 restores the automatic choice.  Process-wide; not thread-safe
- * against concurrent GEMM calls.  Results do not depend on it.
- */
-int gpusq_set_block_tokens(int block_t);
-
 #ifdef __cplusplus
 }
 #endif

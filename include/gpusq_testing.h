@@ -1,0 +1,30 @@
+/*
+ * gpusq -- hooks for the test suite.  NOT part of the library's interface: a
+ * program that uses libgpusq.so has no reason to call these (the paper has no
+ * counterpart).  They exist so that the parity tests can drive the GEMM
+ * kernels through every tile height and through mixed tile heights on small
+ * shapes; results never depend on them.
+ *
+ * Both settings are process-wide atomics read by every later gpusq_spgemm_i8 /
+ * gpusq_gemm_i8_dense / gpusq_spgemm_f16 call of the process, from any thread;
+ * they are meant to be set while no other thread is issuing GEMM calls.
+ */
+#ifndef GPUSQ_TESTING_H
+#define GPUSQ_TESTING_H
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Tokens per output tile: a multiple of 32 in [32, 224], all tiles of that
+ * height; 0 restores the automatic choice (also of the mix below). */
+int gpusq_set_block_tokens(int block_t);
+
+/* Mixed heights: the first n_big token tiles block_t tokens high (block_t a
+ * multiple of 32 in [64, 224]), the rest block_t - 32, as many as cover M. */
+int gpusq_set_tile_mix(int block_t, int n_big);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GPUSQ_TESTING_H */

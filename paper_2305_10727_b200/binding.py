@@ -24,7 +24,7 @@ SCALE_COMPUTE, SCALE_GIVEN = 0, 1
 EXPORTS = (
     "gpusq_status_string", "gpusq_prune24", "gpusq_quant_weight", "gpusq_compress24",
     "gpusq_decompress24", "gpusq_packed_bytes", "gpusq_pack24", "gpusq_quant_act_workspace",
-    "gpusq_quant_act", "gpusq_quant_act_static", "gpusq_patch_quant", "gpusq_spgemm_i8", "gpusq_gemm_i8_dense", "gpusq_set_block_tokens",
+    "gpusq_quant_act", "gpusq_quant_act_static", "gpusq_patch_quant", "gpusq_spgemm_i8", "gpusq_gemm_i8_dense", "gpusq_set_block_tokens", "gpusq_set_tile_mix",
     "gpusq_compress24_f16", "gpusq_packed_bytes_f16", "gpusq_pack24_f16", "gpusq_spgemm_f16",
 )
 
@@ -66,6 +66,7 @@ def load() -> ctypes.CDLL:
     lib.gpusq_spgemm_i8.argtypes = gemm_args
     lib.gpusq_gemm_i8_dense.argtypes = gemm_args
     lib.gpusq_set_block_tokens.argtypes = [i32]
+    lib.gpusq_set_tile_mix.argtypes = [i32, i32]
     lib.gpusq_compress24_f16.argtypes = [vp, vp, vp, i32, i32, vp]
     lib.gpusq_packed_bytes_f16.argtypes = [i32, i32]
     lib.gpusq_packed_bytes_f16.restype = sz
@@ -260,7 +261,13 @@ def gemm_i8_dense(Xq: torch.Tensor, Wq: torch.Tensor, w_scale=None, x_scale=None
 
 
 def set_block_tokens(block_t: int) -> None:
+    """Test hook (gpusq_testing.h): force the GEMM tile height; 0 = automatic."""
     _check(load().gpusq_set_block_tokens(block_t), "gpusq_set_block_tokens")
+
+
+def set_tile_mix(block_t: int, n_big: int) -> None:
+    """Test hook (gpusq_testing.h): n_big token tiles of block_t tokens, the rest 32 tokens lower."""
+    _check(load().gpusq_set_tile_mix(block_t, n_big), "gpusq_set_tile_mix")
 
 
 # ---- FP16 2:4 sparse model ----

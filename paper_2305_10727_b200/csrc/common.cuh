@@ -5,6 +5,7 @@
 #include <stdint.h>
 
 #include "gpusq.h"
+#include "gpusq_testing.h"
 
 namespace gpusq {
 

@@ -43,6 +43,7 @@
 #include <cuda.h>
 #include <cuda_fp16.h>
 
+#include <atomic>
 #include <mutex>
 
 #include "common.cuh"
@@ -114,7 +115,8 @@ struct GemmParams {
     int64_t M;
     int N;
     int K;
-    int block_t;
+    int block_t;    // tokens per tile, a multiple of 32: the height of the first n_big token tiles
+    int n_big;      // token tiles of full height; the token tiles after them are 32 tokens lower
     int act;
     int out_type;
     int pair_cols;  // feature columns of 256 that are worked on as ordinary pair tiles
@@ -124,29 +126,61 @@ struct GemmParams {
     int oob_row;    // a row coordinate beyond the weight tensor: loads from there fill with zeros
 };
 
-// Where a tile sits.  Normally a pair shares `block_t` tokens and CTA `rank` owns 128 of the pair's
-// 256 features.  When the last column of features is at most 128 wide (N mod 256 in 1..128: every
+// Where a tile sits.  Normally a pair shares `h` tokens and CTA `rank` owns 128 of the pair's 256
+// features.  Token tiles come in two heights so that the number of tiles can be made to fit the
+// number of CTA pairs (the last wave of a persistent launch is otherwise partly empty): the first
+// n_big token tiles are block_t tokens high, the ones after them block_t - 32.
+// When the last column of features is at most 128 wide (N mod 256 in 1..128: every
 // layer of at most 128 features, and e.g. N = 384) that would leave the second CTA without output,
 // so that column is worked on in "twin" tiles: each CTA owns the column's features of its OWN
 // `block_t` tokens, and the pair's MMA runs over the k blocks twice, first against the token tile of
 // CTA 0 with the weight block in CTA 0's shared memory and zeros in CTA 1's, then against CTA 1's
 // tokens the other way round, so each CTA's accumulator ends up with W times its own tokens.
-// Ordinary tiles come first (feature column fastest), twin tiles after them.  Returns whether the
-// tile is a twin tile.
+// Ordinary tiles come first (feature column fastest), twin tiles after them.
 // kTwin = false (no twin column in this launch) compiles the test away.
 template <bool kTwin>
-__device__ __forceinline__ bool tile_origin(const GemmParams &p, int tile, int rank, int &n0, int64_t &m0)
-{
-    if (kTwin && tile >= p.pair_tiles) {
-        n0 = p.twin_n0;
-        m0 = ((int64_t)(tile - p.pair_tiles) * 2 + rank) * p.block_t;
-        return true;
+struct TileWalk {
+    int tile;       // cluster_id, cluster_id + num_clusters, ...
+    int tn, tm;     // feature column and token tile of an ordinary tile, kept incrementally (no division per tile)
+    int step_n, step_m;
+
+    __device__ __forceinline__ TileWalk(const GemmParams &p, int cluster_id, int num_clusters)
+    {
+        const int cols = p.pair_cols > 0 ? p.pair_cols : 1;
+        tile = cluster_id;
+        tn = cluster_id % cols;
+        tm = cluster_id / cols;
+        step_n = num_clusters % cols;
+        step_m = num_clusters / cols;
     }
-    const int tn = tile % p.pair_cols, tm = tile / p.pair_cols;
-    n0 = tn * kPairF + rank * kBlockF;
-    m0 = (int64_t)tm * p.block_t;
-    return false;
-}
+    __device__ __forceinline__ void next(const GemmParams &p, int num_clusters)
+    {
+        tile += num_clusters;
+        tn += step_n;
+        tm += step_m;
+        if (tn >= p.pair_cols) {
+            tn -= p.pair_cols;
+            ++tm;
+        }
+    }
+    __device__ __forceinline__ bool twin(const GemmParams &p) const { return kTwin && tile >= p.pair_tiles; }
+    // the tile is one of the lower ones (token tiles from n_big on)
+    __device__ __forceinline__ bool low(const GemmParams &p) const { return !twin(p) && tm >= p.n_big; }
+    // first feature and first token of CTA `rank`'s part, and the tile's height in tokens
+    __device__ __forceinline__ void origin(const GemmParams &p, int rank, int &n0, int64_t &m0, int &h) const
+    {
+        if (twin(p)) {
+            n0 = p.twin_n0;
+            m0 = ((int64_t)(tile - p.pair_tiles) * 2 + rank) * p.block_t;
+            h = p.block_t;
+            return;
+        }
+        n0 = tn * kPairF + rank * kBlockF;
+        const int below = tm - p.n_big;                 // > 0: that many lower tiles precede this one
+        h = below >= 0 ? p.block_t - 32 : p.block_t;
+        m0 = (int64_t)tm * p.block_t - (below > 0 ? (int64_t)below * 32 : 0);
+    }
+};
 
 // A wait of this CTA expired: raise the abort flag in both CTAs of the pair and record where.
 __device__ __forceinline__ void report_timeout(const GemmParams &p, Ctl *ctl, int tile, int role, int stage)
@@ -168,12 +202,13 @@ __device__ __forceinline__ void report_timeout(const GemmParams &p, Ctl *ctl, in
 // to t = 4.3, so g keeps a relative accuracy of ~8e-6 wherever the binary16 result is a normal
 // number, negative tail included; beyond, where the result is subnormal, the fit is looser but stays
 // within a fraction of the subnormal spacing).  Beyond t = 6, g < 2^-25.
-// The coefficients are duplicated so that a packed FP32 instruction can take a pair straight from the
-// constant bank.
+// The polynomial is written in u = -t (odd coefficients negated), so that the result is one fused
+// multiply-add max(y, 0) + u * 2^p.  The coefficients are duplicated so that a packed FP32
+// instruction can take a pair straight from the constant bank.
 __constant__ float2 kGeluC[7] = {
-    {-1.000003934e+00f, -1.000003934e+00f}, {-1.151062012e+00f, -1.151062012e+00f},
-    {-4.591387510e-01f, -4.591387510e-01f}, {-5.306138098e-02f, -5.306138098e-02f},
-    {7.939796895e-03f, 7.939796895e-03f},   {-7.468767581e-04f, -7.468767581e-04f},
+    {-1.000003934e+00f, -1.000003934e+00f}, {1.151062012e+00f, 1.151062012e+00f},
+    {-4.591387510e-01f, -4.591387510e-01f}, {5.306138098e-02f, 5.306138098e-02f},
+    {7.939796895e-03f, 7.939796895e-03f},   {7.468767581e-04f, 7.468767581e-04f},
     {3.226381159e-05f, 3.226381159e-05f},
 };
 
@@ -187,13 +222,13 @@ __device__ __forceinline__ float ex2_approx(float x)
 // two values at a time: the polynomial runs on packed FP32 pairs (fma.rn.f32x2)
 __device__ __forceinline__ float2 gelu_pair(float2 y)
 {
-    const float2 t = make_float2(fminf(fabsf(y.x), 6.0f), fminf(fabsf(y.y), 6.0f));
+    const float2 u = make_float2(fmaxf(-fabsf(y.x), -6.0f), fmaxf(-fabsf(y.y), -6.0f));
     float2 r = kGeluC[6];
 #pragma unroll
-    for (int d = 5; d >= 0; --d) r = __ffma2_rn(r, t, kGeluC[d]);
-    const float2 g = __fmul2_rn(t, make_float2(ex2_approx(r.x), ex2_approx(r.y)));
-    // max(y, 0) - g
-    return __ffma2_rn(g, make_float2(-1.0f, -1.0f), make_float2(fmaxf(y.x, 0.0f), fmaxf(y.y, 0.0f)));
+    for (int d = 5; d >= 0; --d) r = __ffma2_rn(r, u, kGeluC[d]);
+    // max(y, 0) + u * 2^p
+    return __ffma2_rn(u, make_float2(ex2_approx(r.x), ex2_approx(r.y)),
+                      make_float2(fmaxf(y.x, 0.0f), fmaxf(y.y, 0.0f)));
 }
 
 // FP16 epilogue of one worker warp.  The warp owns 16 tensor-memory lanes (features) and every
@@ -207,7 +242,7 @@ struct EpiF16 {
     Ctl *ctl;
     uint32_t tmem_base, stage0, stg_full0, stg_free0, tmem_empty0, tmem_empty1;
     float x_scale;
-    int warp, lane, rank, cluster_id, num_clusters, tiles_n, num_tiles, block_t;
+    int warp, lane, rank, cluster_id, num_clusters, tiles_n, num_tiles;
 
     // staging-tile ring of this warp's group
     uint32_t buf_addr, full_bar, free_bar, buf_idx, free_parity;
@@ -291,18 +326,17 @@ struct EpiF16 {
         free_bar = stg_free0;
         buf_idx = 0;
         free_parity = 1;                                   // first round: the tiles are free
-        const int chunks = block_t / kChunkT;
         const int64_t M = p->M;
         const int N = p->N;
         const float *w_scale = p->w_scale, *bias = p->bias;
 
         // scale and bias of a tile are fetched one tile ahead: the loads are in flight during a whole tile
         float ws_next[2], bi_next[2];
-        auto fetch = [&](int tile) {
-            int n0;
+        auto fetch = [&](const TileWalk<kTwin> &w) {
+            int n0, unused_h;
             int64_t unused;
-            (void)tile_origin<kTwin>(*p, tile, rank, n0, unused);
-            const bool in = tile < num_tiles && n0 < N;
+            w.origin(*p, rank, n0, unused, unused_h);
+            const bool in = w.tile < num_tiles && n0 < N;
 #pragma unroll
             for (int j = 0; j < 2; ++j) {
                 const int n = n0 + nofs + 8 * j;           // N need not fill the last 128-feature block
@@ -310,12 +344,15 @@ struct EpiF16 {
                 bi_next[j] = (in && n < N && bias) ? __ldg(bias + n) : 0.0f;
             }
         };
-        fetch(cluster_id);
+        TileWalk<kTwin> walk(*p, cluster_id, num_clusters);
+        fetch(walk);
         int local = 0;
-        for (int tile = cluster_id; tile < num_tiles; tile += num_clusters, ++local) {
-            int n0;
+        for (; walk.tile < num_tiles; ++local) {
+            const int tile = walk.tile;
+            int n0, h;
             int64_t m0;
-            (void)tile_origin<kTwin>(*p, tile, rank, n0, m0);
+            walk.origin(*p, rank, n0, m0, h);
+            walk.next(*p, num_clusters);
             const int acc = local & 1;
             const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
             const bool n_valid = n0 < N;                   // the pair's second CTA may lie past the last feature
@@ -325,7 +362,7 @@ struct EpiF16 {
                 sc2[j] = make_float2(sc, sc);
                 bi2[j] = make_float2(bi_next[j], bi_next[j]);
             }
-            fetch(tile + num_clusters);
+            fetch(walk);
             bool to;
             if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->tmem_full[acc]), acc_phase, &ctl->abort_flag, to)) {
                 if (to && lane == 0) report_timeout(*p, ctl, tile, 2, 100 + acc);
@@ -335,7 +372,7 @@ struct EpiF16 {
             int nchunks = 0;
             if (n_valid) {
                 const int64_t left = M - m0;               // > 0
-                nchunks = left >= block_t ? chunks : (int)((left + kChunkT - 1) / kChunkT);
+                nchunks = left >= h ? h / kChunkT : (int)((left + kChunkT - 1) / kChunkT);
             }
             // this warp's chunks of the tile: c0, c0 + 2, ...; the two parity groups swap every tile
             const int c0 = (par + local) & 1;
@@ -373,7 +410,7 @@ struct EpiI8 {
     uint8_t *epi_smem;
     uint32_t tmem_base, tmem_empty0, tmem_empty1;
     float x_scale, out_scale;
-    int warp, lane, rank, cluster_id, num_clusters, tiles_n, num_tiles, block_t;
+    int warp, lane, rank, cluster_id, num_clusters, tiles_n, num_tiles;
 
     __device__ __forceinline__ void release(int acc)
     {
@@ -396,34 +433,36 @@ struct EpiI8 {
         const uint32_t ring0 = ptx::smem_u32(epi_smem + sub * kEpiBufs * kEpiBufBytes);
         const uint32_t full0 = ptx::smem_u32(&ctl->stg_full[sub][0]), free0 = ptx::smem_u32(&ctl->stg_free[sub][0]);
         uint32_t buf_addr = ring0, full_bar = full0, free_bar = free0, buf_idx = 0, free_parity = 1;
-        const int chunks = block_t / kChunkT;
         const int64_t M = p->M;
         const int N = p->N;
         const float *w_scale = p->w_scale, *bias = p->bias;
         const QuantScale qs = make_quant_scale(out_scale);
 
         float ws_next, bi_next;
-        auto fetch = [&](int tile) {
-            int n0;
+        auto fetch = [&](const TileWalk<kTwin> &w) {
+            int n0, unused_h;
             int64_t unused;
-            (void)tile_origin<kTwin>(*p, tile, rank, n0, unused);
+            w.origin(*p, rank, n0, unused, unused_h);
             const int n = n0 + quarter * 32 + lane;
-            const bool in = tile < num_tiles && n < N;
+            const bool in = w.tile < num_tiles && n < N;
             ws_next = in ? __ldg(w_scale + n) : 0.0f;
             bi_next = (in && bias) ? __ldg(bias + n) : 0.0f;
         };
-        fetch(cluster_id);
+        TileWalk<kTwin> walk(*p, cluster_id, num_clusters);
+        fetch(walk);
         int local = 0;
-        for (int tile = cluster_id; tile < num_tiles; tile += num_clusters, ++local) {
-            int n0;
+        for (; walk.tile < num_tiles; ++local) {
+            const int tile = walk.tile;
+            int n0, h;
             int64_t m0;
-            (void)tile_origin<kTwin>(*p, tile, rank, n0, m0);
+            walk.origin(*p, rank, n0, m0, h);
+            walk.next(*p, num_clusters);
             const int acc = local & 1;
             const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
             const bool n_valid = n0 < N;
             const float sc = __fmul_rn(ws_next, x_scale);
             const float2 sc2 = make_float2(sc, sc), bi2 = make_float2(bi_next, bi_next);
-            fetch(tile + num_clusters);
+            fetch(walk);
             bool to;
             if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->tmem_full[acc]), acc_phase, &ctl->abort_flag, to)) {
                 if (to && lane == 0) report_timeout(*p, ctl, tile, 2, 100 + acc);
@@ -433,7 +472,7 @@ struct EpiI8 {
             int nchunks = 0;
             if (n_valid) {
                 const int64_t left = M - m0;
-                nchunks = left >= block_t ? chunks : (int)((left + kChunkT - 1) / kChunkT);
+                nchunks = left >= h ? h / kChunkT : (int)((left + kChunkT - 1) / kChunkT);
             }
             const int c0 = (sub - local) & 3;              // chunk c belongs to the warps with sub == (c + local) % 4
             if (c0 >= nchunks) {
@@ -506,8 +545,8 @@ struct EpiI8 {
 template <bool kSparse, int kOut, bool kHalf = false, bool kTwin = false>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kNumThreads, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-               const __grid_constant__ CUtensorMap map_e, const __grid_constant__ CUtensorMap map_y,
-               const GemmParams p)
+               const __grid_constant__ CUtensorMap map_b2, const __grid_constant__ CUtensorMap map_e,
+               const __grid_constant__ CUtensorMap map_y, const GemmParams p)
 {
     using C = Cfg<kSparse, kHalf>;
     extern __shared__ uint8_t smem_raw[];
@@ -523,13 +562,9 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const uint32_t rank = ptx::cluster_ctarank();            // 0 issues the MMAs of the pair
     const int cluster_id = blockIdx.x >> 1;
     const int num_clusters = gridDim.x >> 1;
-    const int block_t = p.block_t;
-    const int half_t = block_t >> 1;
     const int tiles_n = (p.N + kPairF - 1) / kPairF;
     const int num_tiles = p.num_tiles;
     const int k_blocks = (p.K + kBlockK - 1) / kBlockK;        // k blocks of the layer; a twin tile takes them twice
-    // bytes both CTAs together bring in per stage
-    const uint32_t stage_tx = 2u * (uint32_t)(C::kABytes + C::kBAtoms * half_t * 128 + C::kMetaBytes);
 
     auto a_smem = [&](int s) { return smem + s * C::kStageBytes; };
     auto b_smem = [&](int s) { return smem + s * C::kStageBytes + C::kABytes; };
@@ -554,6 +589,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         ptx::fence_barrier_init();
         ptx::prefetch_tensormap(&map_a);
         ptx::prefetch_tensormap(&map_b);
+        if (p.n_big * p.pair_cols < p.pair_tiles) ptx::prefetch_tensormap(&map_b2);
         if (kSparse) ptx::prefetch_tensormap(&map_e);
         if (kOut != GPUSQ_OUT_I32) ptx::prefetch_tensormap(&map_y);
     }
@@ -580,11 +616,19 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             uint32_t issued = 0;            // bit s: a load into stage s was issued
             uint32_t last_parity = 0;       // bit s: parity of the last phase issued into stage s
             bool ok = true;
-            for (int tile = cluster_id; ok && tile < num_tiles; tile += num_clusters) {
-                const bool twin = kTwin && tile >= p.pair_tiles;
+            for (TileWalk<kTwin> walk(p, cluster_id, num_clusters); ok && walk.tile < num_tiles; walk.next(p, num_clusters)) {
+                const int tile = walk.tile;
+                const bool twin = walk.twin(p);
                 const int tw = tile - p.pair_tiles;                               // index among the twin tiles
-                const int tn = twin ? 0 : tile % p.pair_cols, tm = twin ? 0 : tile / p.pair_cols;
+                const int tn = twin ? 0 : walk.tn;
                 const int num_kb = twin ? 2 * k_blocks : k_blocks;
+                int n0_unused, h;
+                int64_t m0;
+                walk.origin(p, 0, n0_unused, m0, h);                               // token origin of the pair's tile
+                const int half_t = h >> 1;
+                const CUtensorMap *mb = h == p.block_t ? &map_b : &map_b2;         // box height = half the tile's tokens
+                // bytes both CTAs together bring in per stage
+                const uint32_t stage_tx = 2u * (uint32_t)(C::kABytes + C::kBAtoms * half_t * 128 + C::kMetaBytes);
                 for (int ks = 0; ks < num_kb; ++ks) {
                     // twin tiles: pass `seg` of the k blocks runs against the token tile of CTA `seg`, whose
                     // weights sit in that CTA only (the other one loads zeros from beyond the tensor)
@@ -592,7 +636,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     const int kb = ks - seg * k_blocks;
                     const int w0 = twin ? p.twin_n0 : tn * kPairF + (int)rank * kBlockF;   // first weight row wanted
                     const int f0 = (twin && seg != (int)rank) ? p.oob_row : w0;          // first weight row loaded
-                    const int t0 = (twin ? (2 * tw + seg) * block_t : tm * block_t) + (int)rank * half_t;
+                    const int t0 = (twin ? (2 * tw + seg) * p.block_t : (int)m0) + (int)rank * half_t;
                     bool to;
                     if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->empty[stage]), phase ^ 1u, abort_flag, to)) {
                         if (to) report_timeout(p, ctl, tile, 0, stage);
@@ -606,11 +650,11 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                                           kb * (kHalf ? 128 : kSparse ? 64 : 128), f0);
                     if (kHalf) {
                         // 128 binary16 columns = two tiles of 128 bytes per token row
-                        ptx::tma_load_2d_pair(ptx::smem_u32(b_smem(stage)), &map_b, bar, kb * 256, t0);
-                        ptx::tma_load_2d_pair(ptx::smem_u32(b_smem(stage)) + (uint32_t)(half_t * 128), &map_b, bar,
+                        ptx::tma_load_2d_pair(ptx::smem_u32(b_smem(stage)), mb, bar, kb * 256, t0);
+                        ptx::tma_load_2d_pair(ptx::smem_u32(b_smem(stage)) + (uint32_t)(half_t * 128), mb, bar,
                                               kb * 256 + 128, t0);
                     } else {
-                        ptx::tma_load_2d_pair(ptx::smem_u32(b_smem(stage)), &map_b, bar, kb * kBlockK, t0);
+                        ptx::tma_load_2d_pair(ptx::smem_u32(b_smem(stage)), mb, bar, kb * kBlockK, t0);
                     }
                     if (kSparse) {
                         // 2 KB metadata block of (feature tile, k block) = 8 rows of 256 bytes
@@ -639,12 +683,17 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     } else if (warp == 1) {
         // ---------------------------------------------------------- MMA issuer
         if (rank == 0 && ptx::elect_one()) {
-            const uint32_t idesc = kHalf ? ptx::make_idesc_f16_sparse(kPairF, block_t) : ptx::make_idesc_i8(kPairF, block_t, kSparse);
+            const uint32_t idesc_big = kHalf ? ptx::make_idesc_f16_sparse(kPairF, p.block_t)
+                                             : ptx::make_idesc_i8(kPairF, p.block_t, kSparse);
+            const uint32_t idesc_low = kHalf ? ptx::make_idesc_f16_sparse(kPairF, p.block_t - 32)
+                                             : ptx::make_idesc_i8(kPairF, p.block_t - 32, kSparse);
             int stage = 0;
             uint32_t phase = 0;
             int local = 0;
             bool ok = true;
-            for (int tile = cluster_id; ok && tile < num_tiles; tile += num_clusters, ++local) {
+            for (TileWalk<kTwin> walk(p, cluster_id, num_clusters); ok && walk.tile < num_tiles;
+                 walk.next(p, num_clusters), ++local) {
+                const int tile = walk.tile;
                 const int acc = local & 1;
                 const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
                 bool to;
@@ -655,7 +704,11 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 }
                 ptx::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kAccStride);
-                const int num_kb = (kTwin && tile >= p.pair_tiles) ? 2 * k_blocks : k_blocks;
+                const int num_kb = walk.twin(p) ? 2 * k_blocks : k_blocks;
+                // a tile of lower height (the token tiles from n_big on) takes the narrower instruction
+                const bool low = walk.low(p);
+                const uint32_t idesc = low ? idesc_low : idesc_big;
+                const int half_t = (low ? p.block_t - 32 : p.block_t) >> 1;
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->full[stage]), phase, abort_flag, to)) {
                         if (to) report_timeout(p, ctl, tile, 1, stage);
@@ -709,18 +762,19 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // tiles back to the epilogue warps once the stores have read them.
         if (kOut == GPUSQ_OUT_F16 && ptx::elect_one()) {
             const int fgroup = warp - kStoreWarp0;         // features [64 fgroup, 64 fgroup + 64) of the CTA's 128
-            const int chunks = block_t / kChunkT;
             uint32_t filled0 = 0, filled1 = 0;             // staging tiles stored so far, per chunk parity group
             uint32_t prev1 = 0, prev2 = 0;                 // free barriers of the last two stores (0 = none)
             int local = 0;
             bool ok = true;
-            for (int tile = cluster_id; ok && tile < num_tiles; tile += num_clusters, ++local) {
-                int n0;
+            for (TileWalk<kTwin> walk(p, cluster_id, num_clusters); ok && walk.tile < num_tiles;
+                 walk.next(p, num_clusters), ++local) {
+                const int tile = walk.tile;
+                int n0, h;
                 int64_t m0;
-                (void)tile_origin<kTwin>(p, tile, (int)rank, n0, m0);
+                walk.origin(p, (int)rank, n0, m0, h);
                 if (n0 >= p.N) continue;
                 const int64_t left = p.M - m0;
-                const int nchunks = left >= block_t ? chunks : (int)((left + kChunkT - 1) / kChunkT);
+                const int nchunks = left >= h ? h / kChunkT : (int)((left + kChunkT - 1) / kChunkT);
                 for (int c = 0; c < nchunks; ++c) {
                     const int par = (c + local) & 1;       // the group of warps that fills this chunk
                     const int gi = fgroup * 2 + par;
@@ -751,18 +805,19 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             // INT8 output: staging tiles hold all 128 features of a chunk; rings 0..3 belong to the warps
             // with that chunk index modulo 4 (rotating per tile); this lane serves rings `odd` and `odd + 2`
             const int odd = warp - kStoreWarp0;
-            const int chunks = block_t / kChunkT;
             uint32_t filled_lo = 0, filled_hi = 0;         // staging tiles stored so far from ring odd / odd + 2
             uint32_t prev1 = 0, prev2 = 0;
             int local = 0;
             bool ok = true;
-            for (int tile = cluster_id; ok && tile < num_tiles; tile += num_clusters, ++local) {
-                int n0;
+            for (TileWalk<kTwin> walk(p, cluster_id, num_clusters); ok && walk.tile < num_tiles;
+                 walk.next(p, num_clusters), ++local) {
+                const int tile = walk.tile;
+                int n0, h;
                 int64_t m0;
-                (void)tile_origin<kTwin>(p, tile, (int)rank, n0, m0);
+                walk.origin(p, (int)rank, n0, m0, h);
                 if (n0 >= p.N) continue;
                 const int64_t left = p.M - m0;
-                const int nchunks = left >= block_t ? chunks : (int)((left + kChunkT - 1) / kChunkT);
+                const int nchunks = left >= h ? h / kChunkT : (int)((left + kChunkT - 1) / kChunkT);
                 for (int c = 0; c < nchunks; ++c) {
                     const int ring = (c + local) & 3;
                     if ((ring & 1) != odd) continue;
@@ -818,7 +873,6 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             e.num_clusters = num_clusters;
             e.tiles_n = tiles_n;
             e.num_tiles = num_tiles;
-            e.block_t = block_t;
             if (p.act == GPUSQ_ACT_GELU)
                 e.template run<true>();
             else
@@ -840,7 +894,6 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             e.num_clusters = num_clusters;
             e.tiles_n = tiles_n;
             e.num_tiles = num_tiles;
-            e.block_t = block_t;
             if (p.act == GPUSQ_ACT_GELU)
                 e.template run<true>();
             else
@@ -848,10 +901,11 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         } else {
             // raw INT32 accumulators (for bit-exact comparison): plain coalesced stores; the four warps
             // of a quarter take every fourth 16-token chunk
-            for (int tile = cluster_id; tile < num_tiles; tile += num_clusters, ++local) {
-                int n0;
+            for (TileWalk<kTwin> walk(p, cluster_id, num_clusters); walk.tile < num_tiles; walk.next(p, num_clusters), ++local) {
+                const int tile = walk.tile;
+                int n0, h;
                 int64_t m0;
-                (void)tile_origin<kTwin>(p, tile, (int)rank, n0, m0);
+                walk.origin(p, (int)rank, n0, m0, h);
                 const int acc = local & 1;
                 const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
                 const bool n_valid = n0 < p.N;
@@ -863,7 +917,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 }
                 ptx::tc_fence_after();
                 const uint32_t tbase = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * kAccStride);
-                for (int c = (warp - 2) >> 2; c < block_t / 16 && n_valid; c += kEpiWarps / 4) {
+                for (int c = (warp - 2) >> 2; c < h / 16 && n_valid; c += kEpiWarps / 4) {
                     if (m0 + c * 16 >= p.M) break;
                     uint32_t r[16];
                     ptx::tmem_ld_32x32b_x16(tbase + (uint32_t)(c * 16), r);
@@ -940,28 +994,137 @@ static bool make_map_y_f16(CUtensorMap *map, void *base, uint64_t M, uint64_t N)
            CUDA_SUCCESS;
 }
 
-static int g_block_t_override = 0;
+// testing hooks (gpusq_testing.h): a forced tile height, and a forced number of full-height token tiles
+static std::atomic<int> g_block_t_override{0};
+static std::atomic<int> g_n_big_override{-1};
 
-// Tokens per tile: a multiple of 32 up to 224 that minimises waves x time per tile.  Per tile and CTA
-// the shared memory moves, per 128-wide k block, 128 bytes per token (activations written and read)
-// plus a fixed ~20 KB for the weight block (as much as 160 tokens), and the epilogue's staging costs
-// as much as four k blocks per token: time per tile ~ (kb + 4) * block_t + 160 * kb.
-static int choose_block_t(int64_t M, int tiles_n, int clusters, int K)
+// How the token axis is cut into tiles: tok_tiles token tiles, the first n_big of them block_t tokens
+// high, the others block_t - 32.
+struct TilePlan {
+    int block_t, n_big, tok_tiles;
+};
+
+// Relative time of one tile of h tokens over kb 128-wide k blocks.  Per tile and CTA the shared memory
+// moves, per k block, 128 bytes per token (activations written and read) plus a fixed ~20 KB for the
+// weight block (as much as 160 tokens), and the epilogue's staging costs as much as four k blocks per
+// token: time per tile ~ (kb + 4) * h + 160 * kb.
+static double tile_cost(double kb, int64_t h) { return (kb + 4.0) * (double)h + 160.0 * kb; }
+
+// Time until the last cluster is done when cluster c works on tiles c, c + clusters, ...: the pair
+// tiles (token tile major, pair_cols feature columns each) first, then the twin tiles of a last
+// narrow feature column (two token tiles of block_t each, the k blocks taken twice).
+static double makespan(const TilePlan &t, int64_t M, int pair_cols, bool twin_col, int clusters, double kb)
 {
-    if (g_block_t_override) return g_block_t_override;
+    double load[148] = {};
+    const int C = clusters < 148 ? clusters : 148;
+    int64_t i = 0;
+    for (int tm = 0; tm < t.tok_tiles; ++tm) {
+        const int low = tm - t.n_big;
+        const int64_t h = low >= 0 ? t.block_t - 32 : t.block_t;
+        const int64_t m0 = (int64_t)tm * t.block_t - (low > 0 ? (int64_t)low * 32 : 0);
+        const double c = tile_cost(kb, M - m0 < h ? M - m0 : h);
+        for (int tn = 0; tn < pair_cols; ++tn, ++i) load[i % C] += c;
+    }
+    if (twin_col) {
+        const int64_t twins = ceil_div(M, 2 * (int64_t)t.block_t);
+        for (int64_t w = 0; w < twins; ++w, ++i) load[i % C] += tile_cost(2.0 * kb, t.block_t);
+    }
+    double worst = 0.0;
+    for (int c = 0; c < C; ++c) worst = load[c] > worst ? load[c] : worst;
+    return worst;
+}
+
+// Tile heights for a launch.  Uniform tiles leave the last wave of the persistent launch partly
+// empty whenever the tile count is not close to a multiple of the number of clusters (171 tiles on
+// 74 clusters: three waves for 2.3 waves of work); mixing two heights 32 tokens apart gives a tile
+// count that fits.  Searched only while the launch has few waves (beyond that the last wave weighs
+// little and uniform tiles of the best height are taken); the result is remembered per shape.
+static TilePlan plan_tiles(int64_t M, int pair_cols, bool twin_col, int clusters, int K)
+{
     const double kb = (double)ceil_div(K, kBlockK);
-    int best = kMaxBlockT;
+    const int forced = g_block_t_override.load(std::memory_order_relaxed);
+    const int forced_big = g_n_big_override.load(std::memory_order_relaxed);
+    if (forced) {
+        TilePlan t = {forced, (int)ceil_div(M, forced), (int)ceil_div(M, forced)};
+        if (forced_big >= 0 && forced >= 64 && pair_cols > 0) {
+            // as many full-height tiles as asked for (at most what covers M), lower ones for the rest
+            const int64_t nb = forced_big < ceil_div(M, forced) ? forced_big : ceil_div(M, forced);
+            const int64_t rest = M - nb * forced;
+            t.n_big = (int)nb;
+            t.tok_tiles = (int)(nb + (rest > 0 ? ceil_div(rest, forced - 32) : 0));
+        }
+        return t;
+    }
+    struct Entry {
+        int64_t M;
+        int pair_cols, twin, clusters, K;
+        TilePlan plan;
+    };
+    static std::mutex mu;
+    static Entry cache[64];
+    static int used = 0, next = 0;
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        for (int i = 0; i < used; ++i)
+            if (cache[i].M == M && cache[i].pair_cols == pair_cols && cache[i].twin == (int)twin_col &&
+                cache[i].clusters == clusters && cache[i].K == K)
+                return cache[i].plan;
+    }
+    TilePlan best = {kMaxBlockT, 0, 0};
     double best_cost = 1e300;
+    auto consider = [&](const TilePlan &t) {
+        const double c = makespan(t, M, pair_cols, twin_col, clusters, kb);
+        if (c < best_cost * 0.999) {
+            best_cost = c;
+            best = t;
+        }
+    };
     for (int bt = kMaxBlockT; bt >= 32; bt -= 32) {
-        const int64_t tiles = (int64_t)tiles_n * ceil_div(M, bt);
-        const int64_t waves = ceil_div(tiles, clusters);
-        const double cost = (double)waves * ((kb + 4.0) * bt + 160.0 * kb);
-        if (cost < best_cost * 0.999) {
-            best_cost = cost;
-            best = bt;
+        const int64_t t_min = ceil_div(M, bt);
+        if (t_min > 0x7FFFFFF) continue;
+        consider({bt, (int)t_min, (int)t_min});                            // uniform
+        if (bt < 64 || pair_cols == 0 || t_min * pair_cols > 16 * (int64_t)clusters) continue;
+        const int64_t t_max = ceil_div(M, bt - 32);
+        for (int64_t T = t_min; T < t_max; ++T) {
+            // fewest full-height tiles with which T tiles cover M
+            const int64_t need = M - T * (bt - 32);
+            const int64_t nb = need > 0 ? ceil_div(need, 32) : 0;
+            if (nb > T) continue;
+            consider({bt, (int)nb, (int)T});
         }
     }
+    std::lock_guard<std::mutex> lock(mu);
+    cache[next] = {M, pair_cols, (int)twin_col, clusters, K, best};
+    next = (next + 1) % 64;
+    used = used < 64 ? used + 1 : 64;
     return best;
+}
+
+// Fills the tiling fields of the parameters; false when the tile count does not fit 31 bits.
+static bool set_tiling(GemmParams &p, int64_t M, int N, int K_cost, int clusters)
+{
+    const int tiles_n = (N + kPairF - 1) / kPairF;
+    // a last feature column of at most 128 features is worked on in twin tiles (see TileWalk)
+    const bool twin_col = N - (tiles_n - 1) * kPairF <= kBlockF && M < 0x7FFFFFFF - 4 * kMaxBlockT;
+    p.pair_cols = twin_col ? tiles_n - 1 : tiles_n;
+    TilePlan t;
+    if (p.pair_cols == 0) {
+        // twin tiles only: each cluster takes two token tiles and the k blocks twice
+        t = plan_tiles(ceil_div(M, 2), 1, false, clusters, 2 * K_cost);
+        t = {t.block_t, 0, 0};
+    } else {
+        t = plan_tiles(M, p.pair_cols, twin_col, clusters, K_cost);
+    }
+    p.block_t = t.block_t;
+    p.n_big = t.n_big;
+    const int64_t pair_tiles = (int64_t)p.pair_cols * t.tok_tiles;
+    const int64_t tiles = pair_tiles + (twin_col ? ceil_div(M, 2 * (int64_t)t.block_t) : 0);
+    if (tiles > 0x7FFFFFFF) return false;
+    p.pair_tiles = (int)pair_tiles;
+    p.num_tiles = (int)tiles;
+    p.twin_n0 = p.pair_cols * kPairF;
+    p.oob_row = round_up(N, kPairF);  // beyond the packed rows (N rounded up) and the plain ones (N) alike
+    return true;
 }
 
 // SM pairs that can hold one cluster of this kernel each, per device (0 = unknown yet)
@@ -988,6 +1151,72 @@ static int max_clusters(int sms)
     return cached[dev];
 }
 
+// The kernels need more dynamic shared memory than the default limit; the attribute is per device.
+template <typename F>
+static bool allow_smem(F kernel, int bytes)
+{
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess;
+}
+
+// once per device and operand kind (0 sparse INT8, 1 dense INT8, 2 sparse FP16)
+static bool prepare_device(int kind)
+{
+    static std::mutex mu;
+    static uint8_t done[64][3] = {};       // 1 = set, 2 = failed
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+    std::lock_guard<std::mutex> lock(mu);
+    if (done[dev][kind] == 0) {
+        bool ok = true;
+        if (kind == 0) {
+            const int b = Cfg<true>::kSmemBytes;
+            ok = allow_smem(gemm_i8_kernel<true, GPUSQ_OUT_F16>, b) && allow_smem(gemm_i8_kernel<true, GPUSQ_OUT_I8>, b) &&
+                 allow_smem(gemm_i8_kernel<true, GPUSQ_OUT_I32>, b) &&
+                 allow_smem(gemm_i8_kernel<true, GPUSQ_OUT_F16, false, true>, b) &&
+                 allow_smem(gemm_i8_kernel<true, GPUSQ_OUT_I8, false, true>, b) &&
+                 allow_smem(gemm_i8_kernel<true, GPUSQ_OUT_I32, false, true>, b);
+        } else if (kind == 1) {
+            const int b = Cfg<false>::kSmemBytes;
+            ok = allow_smem(gemm_i8_kernel<false, GPUSQ_OUT_F16>, b) && allow_smem(gemm_i8_kernel<false, GPUSQ_OUT_I8>, b) &&
+                 allow_smem(gemm_i8_kernel<false, GPUSQ_OUT_I32>, b) &&
+                 allow_smem(gemm_i8_kernel<false, GPUSQ_OUT_F16, false, true>, b) &&
+                 allow_smem(gemm_i8_kernel<false, GPUSQ_OUT_I8, false, true>, b) &&
+                 allow_smem(gemm_i8_kernel<false, GPUSQ_OUT_I32, false, true>, b);
+        } else {
+            const int b = Cfg<true, true>::kSmemBytes;
+            ok = allow_smem(gemm_i8_kernel<true, GPUSQ_OUT_F16, true>, b) && allow_smem(gemm_i8_kernel<true, GPUSQ_OUT_I32, true>, b) &&
+                 allow_smem(gemm_i8_kernel<true, GPUSQ_OUT_F16, true, true>, b) &&
+                 allow_smem(gemm_i8_kernel<true, GPUSQ_OUT_I32, true, true>, b);
+        }
+        if (!ok) (void)cudaGetLastError();
+        done[dev][kind] = ok ? 1 : 2;
+    }
+    return done[dev][kind] == 1;
+}
+
+template <typename Kernel>
+static int launch_on(Kernel kernel, int smem_bytes, const CUtensorMap &map_a, const CUtensorMap &map_b,
+                     const CUtensorMap &map_b2, const CUtensorMap &map_e, const CUtensorMap &map_y,
+                     const GemmParams &p, int clusters, void *stream)
+{
+    const int grid = 2 * (p.num_tiles < clusters ? p.num_tiles : clusters);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid, 1, 1);
+    cfg.blockDim = dim3(kNumThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem_bytes;
+    cfg.stream = (cudaStream_t)stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;     // start while the previous kernel drains
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, kernel, map_a, map_b, map_b2, map_e, map_y, p) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return GPUSQ_ERR_CUDA;
+    }
+    return GPUSQ_OK;
+}
+
 template <bool kSparse>
 static int launch_gemm(const int8_t *Xq, const void *Wsrc, const float *w_scale, const float *x_scale,
                        const float *bias, int act, int out_type, const float *out_scale, void *Y, int64_t M,
@@ -1003,35 +1232,27 @@ static int launch_gemm(const int8_t *Xq, const void *Wsrc, const float *w_scale,
     if ((out_type == GPUSQ_OUT_F16 && N % 8) || (out_type == GPUSQ_OUT_I8 && N % 16)) return GPUSQ_ERR_SHAPE;
     if (!aligned(Xq, 16) || !aligned(Wsrc, 16) || !aligned(Y, 16)) return GPUSQ_ERR_ALIGN;
     if (int st = check_arch()) return st;
-
-    static std::once_flag attr_once;
-    static cudaError_t attr_err = cudaSuccess;
-    std::call_once(attr_once, [] {
-        const void *kernels[12] = {
-            (const void *)gemm_i8_kernel<true, GPUSQ_OUT_F16>,  (const void *)gemm_i8_kernel<true, GPUSQ_OUT_I8>,
-            (const void *)gemm_i8_kernel<true, GPUSQ_OUT_I32>,
-            (const void *)gemm_i8_kernel<true, GPUSQ_OUT_F16, false, true>,
-            (const void *)gemm_i8_kernel<true, GPUSQ_OUT_I8, false, true>,
-            (const void *)gemm_i8_kernel<true, GPUSQ_OUT_I32, false, true>,
-            (const void *)gemm_i8_kernel<false, GPUSQ_OUT_F16>, (const void *)gemm_i8_kernel<false, GPUSQ_OUT_I8>,
-            (const void *)gemm_i8_kernel<false, GPUSQ_OUT_I32>,
-            (const void *)gemm_i8_kernel<false, GPUSQ_OUT_F16, false, true>,
-            (const void *)gemm_i8_kernel<false, GPUSQ_OUT_I8, false, true>,
-            (const void *)gemm_i8_kernel<false, GPUSQ_OUT_I32, false, true>};
-        for (int k = 0; k < 12 && attr_err == cudaSuccess; ++k)
-            attr_err = cudaFuncSetAttribute(kernels[k], cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            k < 6 ? Cfg<true>::kSmemBytes : Cfg<false>::kSmemBytes);
-    });
-    if (attr_err != cudaSuccess) return GPUSQ_ERR_CUDA;
+    if (!prepare_device(kSparse ? 0 : 1)) return GPUSQ_ERR_CUDA;
 
     const int sms = num_sms();
     const int clusters = max_clusters<kSparse>(sms);
     if (clusters <= 0) return GPUSQ_ERR_CUDA;
-    const int tiles_n = (N + kPairF - 1) / kPairF;
-    // a last feature column of at most 128 features is worked on in twin tiles (see tile_origin)
-    const bool twin_col = N - (tiles_n - 1) * kPairF <= kBlockF && M < 0x7FFFFFFF - 4 * kMaxBlockT;
-    const int block_t = (twin_col && tiles_n == 1) ? choose_block_t(ceil_div(M, 2), 1, clusters, 2 * K)
-                                                   : choose_block_t(M, tiles_n, clusters, K);
+
+    GemmParams p;
+    p.w_scale = w_scale;
+    p.x_scale = x_scale;
+    p.bias = bias;
+    p.out_scale = out_scale;
+    p.Y = Y;
+    p.status = status_buf;
+    p.M = M;
+    p.N = N;
+    p.K = K;
+    p.act = act;
+    p.out_type = out_type;
+    if (!set_tiling(p, M, N, K, clusters)) return GPUSQ_ERR_SHAPE;
+    const bool twin_col = p.pair_tiles < p.num_tiles;
+    const bool mixed = p.block_t >= 64;      // the lower height exists
     const int Kp = round_up(K, 128), Np = round_up(N, kPairF);
 
     CUtensorMap map_a, map_b;
@@ -1040,8 +1261,12 @@ static int launch_gemm(const int8_t *Xq, const void *Wsrc, const float *w_scale,
         ok = make_map_u8(&map_a, Wsrc, (uint64_t)Np, (uint64_t)Kp / 2, 64, kBlockF, CU_TENSOR_MAP_SWIZZLE_64B);
     else
         ok = make_map_u8(&map_a, Wsrc, (uint64_t)N, (uint64_t)K, 128, kBlockF, CU_TENSOR_MAP_SWIZZLE_128B);
-    ok = ok && make_map_u8(&map_b, Xq, (uint64_t)M, (uint64_t)K, 128, (uint32_t)(block_t / 2),
+    ok = ok && make_map_u8(&map_b, Xq, (uint64_t)M, (uint64_t)K, 128, (uint32_t)(p.block_t / 2),
                            CU_TENSOR_MAP_SWIZZLE_128B);
+    CUtensorMap map_b2 = map_b;     // the activation box of the lower tiles
+    if (mixed)
+        ok = ok && make_map_u8(&map_b2, Xq, (uint64_t)M, (uint64_t)K, 128, (uint32_t)(p.block_t / 2 - 16),
+                               CU_TENSOR_MAP_SWIZZLE_128B);
     CUtensorMap map_e = map_b;      // placeholder unless the weight is sparse
     if (kSparse) {
         // metadata blocks of 2 KB, viewed as 8 rows of 256 bytes each
@@ -1056,55 +1281,16 @@ static int launch_gemm(const int8_t *Xq, const void *Wsrc, const float *w_scale,
         ok = ok && make_map_u8(&map_y, Y, (uint64_t)M, (uint64_t)N, 128, (uint32_t)kChunkT, CU_TENSOR_MAP_SWIZZLE_128B);
     if (!ok) return GPUSQ_ERR_CUDA;
 
-    GemmParams p;
-    p.w_scale = w_scale;
-    p.x_scale = x_scale;
-    p.bias = bias;
-    p.out_scale = out_scale;
-    p.Y = Y;
-    p.status = status_buf;
-    p.M = M;
-    p.N = N;
-    p.K = K;
-    p.block_t = block_t;
-    p.act = act;
-    p.out_type = out_type;
-    p.pair_cols = twin_col ? tiles_n - 1 : tiles_n;
-    const int64_t pair_tiles = (int64_t)p.pair_cols * ceil_div(M, block_t);
-    const int64_t tiles = pair_tiles + (twin_col ? ceil_div(M, 2 * (int64_t)block_t) : 0);
-    if (tiles > 0x7FFFFFFF) return GPUSQ_ERR_SHAPE;
-    p.pair_tiles = (int)pair_tiles;
-    p.num_tiles = (int)tiles;
-    p.twin_n0 = p.pair_cols * kPairF;
-    p.oob_row = Np;                 // beyond the packed rows (Np) and the plain ones (N) alike
-
-    const int grid = 2 * (int)(tiles < clusters ? tiles : clusters);
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)grid, 1, 1);
-    cfg.blockDim = dim3(kNumThreads, 1, 1);
-    cfg.dynamicSmemBytes = C::kSmemBytes;
-    cfg.stream = (cudaStream_t)stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;     // start while the previous kernel drains
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    cudaError_t err;
     // launches without a twin column run the instantiation that has no trace of it
+    const int smem = C::kSmemBytes;
     if (out_type == GPUSQ_OUT_F16)
-        err = twin_col ? cudaLaunchKernelEx(&cfg, gemm_i8_kernel<kSparse, GPUSQ_OUT_F16, false, true>, map_a, map_b, map_e, map_y, p)
-                       : cudaLaunchKernelEx(&cfg, gemm_i8_kernel<kSparse, GPUSQ_OUT_F16>, map_a, map_b, map_e, map_y, p);
-    else if (out_type == GPUSQ_OUT_I8)
-        err = twin_col ? cudaLaunchKernelEx(&cfg, gemm_i8_kernel<kSparse, GPUSQ_OUT_I8, false, true>, map_a, map_b, map_e, map_y, p)
-                       : cudaLaunchKernelEx(&cfg, gemm_i8_kernel<kSparse, GPUSQ_OUT_I8>, map_a, map_b, map_e, map_y, p);
-    else
-        err = twin_col ? cudaLaunchKernelEx(&cfg, gemm_i8_kernel<kSparse, GPUSQ_OUT_I32, false, true>, map_a, map_b, map_e, map_y, p)
-                       : cudaLaunchKernelEx(&cfg, gemm_i8_kernel<kSparse, GPUSQ_OUT_I32>, map_a, map_b, map_e, map_y, p);
-    if (err != cudaSuccess) {
-        (void)cudaGetLastError();
-        return GPUSQ_ERR_CUDA;
-    }
-    return GPUSQ_OK;
+        return twin_col ? launch_on(gemm_i8_kernel<kSparse, GPUSQ_OUT_F16, false, true>, smem, map_a, map_b, map_b2, map_e, map_y, p, clusters, stream)
+                        : launch_on(gemm_i8_kernel<kSparse, GPUSQ_OUT_F16>, smem, map_a, map_b, map_b2, map_e, map_y, p, clusters, stream);
+    if (out_type == GPUSQ_OUT_I8)
+        return twin_col ? launch_on(gemm_i8_kernel<kSparse, GPUSQ_OUT_I8, false, true>, smem, map_a, map_b, map_b2, map_e, map_y, p, clusters, stream)
+                        : launch_on(gemm_i8_kernel<kSparse, GPUSQ_OUT_I8>, smem, map_a, map_b, map_b2, map_e, map_y, p, clusters, stream);
+    return twin_col ? launch_on(gemm_i8_kernel<kSparse, GPUSQ_OUT_I32, false, true>, smem, map_a, map_b, map_b2, map_e, map_y, p, clusters, stream)
+                    : launch_on(gemm_i8_kernel<kSparse, GPUSQ_OUT_I32>, smem, map_a, map_b, map_b2, map_e, map_y, p, clusters, stream);
 }
 
 // The FP16 2:4 sparse layer: binary16 activations as they are, FP32 accumulation, bias, optional GELU.
@@ -1118,41 +1304,11 @@ static int launch_gemm_f16(const void *X, const void *Wpacked, const float *bias
     if (out_type == GPUSQ_OUT_F16 && N % 8) return GPUSQ_ERR_SHAPE;
     if (!aligned(X, 16) || !aligned(Wpacked, 256) || !aligned(Y, 16)) return GPUSQ_ERR_ALIGN;
     if (int st = check_arch()) return st;
-
-    static std::once_flag attr_once;
-    static cudaError_t attr_err = cudaSuccess;
-    std::call_once(attr_once, [] {
-        const void *kernels[4] = {
-            (const void *)gemm_i8_kernel<true, GPUSQ_OUT_F16, true>, (const void *)gemm_i8_kernel<true, GPUSQ_OUT_I32, true>,
-            (const void *)gemm_i8_kernel<true, GPUSQ_OUT_F16, true, true>,
-            (const void *)gemm_i8_kernel<true, GPUSQ_OUT_I32, true, true>};
-        for (int k = 0; k < 4 && attr_err == cudaSuccess; ++k)
-            attr_err = cudaFuncSetAttribute(kernels[k], cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
-    });
-    if (attr_err != cudaSuccess) return GPUSQ_ERR_CUDA;
+    if (!prepare_device(2)) return GPUSQ_ERR_CUDA;
 
     const int sms = num_sms();
     const int clusters = max_clusters<true, true>(sms);
     if (clusters <= 0) return GPUSQ_ERR_CUDA;
-    const int tiles_n = (N + kPairF - 1) / kPairF;
-    const bool twin_col = N - (tiles_n - 1) * kPairF <= kBlockF && M < 0x7FFFFFFF - 4 * kMaxBlockT;
-    // twice the bytes per column
-    const int block_t = (twin_col && tiles_n == 1) ? choose_block_t(ceil_div(M, 2), 1, clusters, 4 * K)
-                                                   : choose_block_t(M, tiles_n, clusters, 2 * K);
-    const int Kp = round_up(K, 128), Np = round_up(N, kPairF);
-
-    // every tensor is described in bytes: kept values [Np, Kp] (Kp / 2 binary16 per row), activations
-    // [M, 2 K], metadata blocks of 2 KB as 8 rows of 256 bytes
-    CUtensorMap map_a, map_b, map_e;
-    bool ok = make_map_u8(&map_a, Wpacked, (uint64_t)Np, (uint64_t)Kp, 128, kBlockF, CU_TENSOR_MAP_SWIZZLE_128B);
-    ok = ok && make_map_u8(&map_b, X, (uint64_t)M, (uint64_t)K * 2, 128, (uint32_t)(block_t / 2),
-                           CU_TENSOR_MAP_SWIZZLE_128B);
-    const uint8_t *meta = reinterpret_cast<const uint8_t *>(Wpacked) + (size_t)Np * Kp;
-    ok = ok && make_map_u8(&map_e, meta, (uint64_t)(Np / 128) * (Kp / 128) * 8, 256, 256, 8,
-                           CU_TENSOR_MAP_SWIZZLE_NONE);
-    CUtensorMap map_y = map_b;      // placeholder unless the output is FP16
-    if (out_type == GPUSQ_OUT_F16) ok = ok && make_map_y_f16(&map_y, Y, (uint64_t)M, (uint64_t)N);
-    if (!ok) return GPUSQ_ERR_CUDA;
 
     GemmParams p;
     p.w_scale = nullptr;            // the epilogue's scale is 1
@@ -1164,41 +1320,36 @@ static int launch_gemm_f16(const void *X, const void *Wpacked, const float *bias
     p.M = M;
     p.N = N;
     p.K = K;
-    p.block_t = block_t;
     p.act = act;
     p.out_type = out_type;
-    p.pair_cols = twin_col ? tiles_n - 1 : tiles_n;
-    const int64_t pair_tiles = (int64_t)p.pair_cols * ceil_div(M, block_t);
-    const int64_t tiles = pair_tiles + (twin_col ? ceil_div(M, 2 * (int64_t)block_t) : 0);
-    if (tiles > 0x7FFFFFFF) return GPUSQ_ERR_SHAPE;
-    p.pair_tiles = (int)pair_tiles;
-    p.num_tiles = (int)tiles;
-    p.twin_n0 = p.pair_cols * kPairF;
-    p.oob_row = Np;
+    if (!set_tiling(p, M, N, 2 * K, clusters)) return GPUSQ_ERR_SHAPE;        // twice the bytes per column
+    const bool twin_col = p.pair_tiles < p.num_tiles;
+    const bool mixed = p.block_t >= 64;
+    const int Kp = round_up(K, 128), Np = round_up(N, kPairF);
 
-    const int grid = 2 * (int)(tiles < clusters ? tiles : clusters);
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)grid, 1, 1);
-    cfg.blockDim = dim3(kNumThreads, 1, 1);
-    cfg.dynamicSmemBytes = C::kSmemBytes;
-    cfg.stream = (cudaStream_t)stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    cudaError_t err;
+    // every tensor is described in bytes: kept values [Np, Kp] (Kp / 2 binary16 per row), activations
+    // [M, 2 K], metadata blocks of 2 KB as 8 rows of 256 bytes
+    CUtensorMap map_a, map_b, map_e;
+    bool ok = make_map_u8(&map_a, Wpacked, (uint64_t)Np, (uint64_t)Kp, 128, kBlockF, CU_TENSOR_MAP_SWIZZLE_128B);
+    ok = ok && make_map_u8(&map_b, X, (uint64_t)M, (uint64_t)K * 2, 128, (uint32_t)(p.block_t / 2),
+                           CU_TENSOR_MAP_SWIZZLE_128B);
+    CUtensorMap map_b2 = map_b;
+    if (mixed)
+        ok = ok && make_map_u8(&map_b2, X, (uint64_t)M, (uint64_t)K * 2, 128, (uint32_t)(p.block_t / 2 - 16),
+                               CU_TENSOR_MAP_SWIZZLE_128B);
+    const uint8_t *meta = reinterpret_cast<const uint8_t *>(Wpacked) + (size_t)Np * Kp;
+    ok = ok && make_map_u8(&map_e, meta, (uint64_t)(Np / 128) * (Kp / 128) * 8, 256, 256, 8,
+                           CU_TENSOR_MAP_SWIZZLE_NONE);
+    CUtensorMap map_y = map_b;      // placeholder unless the output is FP16
+    if (out_type == GPUSQ_OUT_F16) ok = ok && make_map_y_f16(&map_y, Y, (uint64_t)M, (uint64_t)N);
+    if (!ok) return GPUSQ_ERR_CUDA;
+
+    const int smem = C::kSmemBytes;
     if (out_type == GPUSQ_OUT_F16)
-        err = twin_col ? cudaLaunchKernelEx(&cfg, gemm_i8_kernel<true, GPUSQ_OUT_F16, true, true>, map_a, map_b, map_e, map_y, p)
-                       : cudaLaunchKernelEx(&cfg, gemm_i8_kernel<true, GPUSQ_OUT_F16, true>, map_a, map_b, map_e, map_y, p);
-    else
-        err = twin_col ? cudaLaunchKernelEx(&cfg, gemm_i8_kernel<true, GPUSQ_OUT_I32, true, true>, map_a, map_b, map_e, map_y, p)
-                       : cudaLaunchKernelEx(&cfg, gemm_i8_kernel<true, GPUSQ_OUT_I32, true>, map_a, map_b, map_e, map_y, p);
-    if (err != cudaSuccess) {
-        (void)cudaGetLastError();
-        return GPUSQ_ERR_CUDA;
-    }
-    return GPUSQ_OK;
+        return twin_col ? launch_on(gemm_i8_kernel<true, GPUSQ_OUT_F16, true, true>, smem, map_a, map_b, map_b2, map_e, map_y, p, clusters, stream)
+                        : launch_on(gemm_i8_kernel<true, GPUSQ_OUT_F16, true>, smem, map_a, map_b, map_b2, map_e, map_y, p, clusters, stream);
+    return twin_col ? launch_on(gemm_i8_kernel<true, GPUSQ_OUT_I32, true, true>, smem, map_a, map_b, map_b2, map_e, map_y, p, clusters, stream)
+                    : launch_on(gemm_i8_kernel<true, GPUSQ_OUT_I32, true>, smem, map_a, map_b, map_b2, map_e, map_y, p, clusters, stream);
 }
 
 }  // namespace gpusq
@@ -1233,7 +1384,16 @@ int gpusq_gemm_i8_dense(const int8_t *Xq, const int8_t *Wq, const float *w_scale
 int gpusq_set_block_tokens(int block_t)
 {
     if (block_t != 0 && (block_t < 32 || block_t > kMaxBlockT || block_t % 32)) return GPUSQ_ERR_ARG;
-    g_block_t_override = block_t;
+    g_block_t_override.store(block_t, std::memory_order_relaxed);
+    g_n_big_override.store(-1, std::memory_order_relaxed);
+    return GPUSQ_OK;
+}
+
+int gpusq_set_tile_mix(int block_t, int n_big)
+{
+    if (block_t < 64 || block_t > kMaxBlockT || block_t % 32 || n_big < 0) return GPUSQ_ERR_ARG;
+    g_block_t_override.store(block_t, std::memory_order_relaxed);
+    g_n_big_override.store(n_big, std::memory_order_relaxed);
     return GPUSQ_OK;
 }
 

@@ -77,12 +77,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 // thread of the CTA has raised *abort_flag.  Returns false on either; the
 // caller that timed out raises the flag itself.  The common case (the phase
 // is complete already) costs one try and one branch; the retry loop is kept
-// out of line so that it does not bloat the callers' instruction streams, and
-// looks at the flag and the clock only every 32 tries.
+// out of line so that it does not bloat the callers' instruction streams.
+// A retry parks the thread in hardware until the phase completes or the hint
+// time has passed, so a waiting warp issues a few instructions per microsecond
+// and wakes as soon as the barrier flips; the flag and the clock are looked at
+// after every `kTriesPerCheck` expired tries.
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s
-constexpr uint32_t kRetrySleepNs = 100;
-// Up to 32 tries with a short sleep after each failed one, as one tight loop (try, branch, sleep,
-// count): waiting warps should cost the working ones as few issue slots as possible.
+constexpr uint32_t kSuspendHintNs = 1000;
 __device__ __forceinline__ bool mbar_try_wait_32(uint32_t bar, uint32_t parity)
 {
     uint32_t ok;
@@ -92,9 +93,8 @@ __device__ __forceinline__ bool mbar_try_wait_32(uint32_t bar, uint32_t parity)
         ".reg .u32 n;\n"
         "mov.u32 n, 32;\n"
         "TRY_AGAIN:\n"
-        "mbarrier.try_wait.parity.shared::cta.b64 P, [%1], %2;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 P, [%1], %2, %3;\n"
         "@P bra DONE;\n"
-        "nanosleep.u32 %3;\n"
         "sub.u32 n, n, 1;\n"
         "setp.ne.u32 Q, n, 0;\n"
         "@Q bra TRY_AGAIN;\n"
@@ -102,7 +102,7 @@ __device__ __forceinline__ bool mbar_try_wait_32(uint32_t bar, uint32_t parity)
         "selp.u32 %0, 1, 0, P;\n"
         "}\n"
         : "=r"(ok)
-        : "r"(bar), "r"(parity), "r"(kRetrySleepNs)
+        : "r"(bar), "r"(parity), "r"(kSuspendHintNs)
         : "memory");
     return ok != 0;
 }

@@ -162,6 +162,38 @@ def test_spgemm_int32_bit_exact(B, M, N, K, block_t):
     assert np.array_equal(Yd.cpu().numpy(), acc_o)       # same C as the dense GEMM (Fig. 1)
 
 
+@pytest.mark.parametrize("M,N,K,block_t,n_big", [
+    (1000, 512, 256, 96, 3), (1576, 768, 192, 224, 2), (700, 256, 128, 64, 0), (2000, 384, 320, 160, 5),
+    (333, 576, 192, 128, 1), (900, 1024, 64, 192, 100), (12608, 768, 256, 192, 24), (5000, 96, 48, 128, 7)])
+def test_mixed_tile_heights(B, M, N, K, block_t, n_big):
+    # token tiles of two heights in one launch (the first n_big of block_t tokens, the rest 32 lower):
+    # accumulators bit-exact, FP16 + GELU within one ulp, INT8 exact, sparse and dense instruction
+    d, prep, Xq, xs = _prep(7 * M + N + K, M, N, K)
+    acc_o = oracle.spgemm_acc(Xq, prep["vals"], prep["meta"], threads=oracle.host_cores())
+    Y_o = oracle.epilogue(acc_o, prep["w_scale"], xs, d["bias"], act=1, out_type=0, threads=oracle.host_cores())
+    yf = oracle.epilogue(acc_o, prep["w_scale"], xs, d["bias"], act=0, out_type=0).astype(np.float32)
+    out_scale = np.float32(np.abs(yf).max() / 127.0)
+    Q_o = oracle.epilogue(acc_o, prep["w_scale"], xs, d["bias"], act=0, out_type=1, out_scale=out_scale)
+    Wpk = B.pack24(cu(prep["vals"]), cu(prep["meta"]))
+    status = torch.zeros(4, dtype=torch.int32, device="cuda")
+    common = dict(w_scale=cu(prep["w_scale"]), x_scale=cu(np.array([xs], np.float32)), bias=cu(d["bias"]),
+                  status_buf=status)
+    B.set_tile_mix(block_t, n_big)
+    try:
+        acc = B.spgemm_i8(cu(Xq), Wpk, N, out_type=B.OUT_I32, status_buf=status).cpu().numpy()
+        accd = B.gemm_i8_dense(cu(Xq), cu(prep["Wq"]), out_type=B.OUT_I32, status_buf=status).cpu().numpy()
+        Y = B.spgemm_i8(cu(Xq), Wpk, N, act=B.ACT_GELU, out_type=B.OUT_F16, **common).cpu().numpy()
+        Q = B.spgemm_i8(cu(Xq), Wpk, N, act=B.ACT_NONE, out_type=B.OUT_I8,
+                        out_scale=cu(np.array([out_scale], np.float32)), **common).cpu().numpy()
+    finally:
+        B.set_block_tokens(0)
+    assert status.cpu().tolist() == [0, 0, 0, 0]
+    assert np.array_equal(acc, acc_o)
+    assert np.array_equal(accd, acc_o)
+    assert f16_ulp_distance(Y, Y_o).max() <= F16_ULP_TOL
+    assert np.array_equal(Q, Q_o)
+
+
 def test_spgemm_extreme_codes_do_not_overflow(B):
     # every kept code and every activation at +-127, K = 5120: |acc| = 127^2 * K / 2
     M, N, K = 40, 128, 5120
