@@ -128,11 +128,21 @@ int gpusq_pack24(const int8_t *vals, const uint8_t *meta, void *Wpacked, int N, 
  *     of any size, so one buffer serves a whole stream of calls.  Calls that
  *     can overlap on the GPU need separate workspaces.
  *   GPUSQ_SCALE_COMPUTE runs as one cooperative launch whose CTAs meet at a
- *   grid-wide barrier; its wait is bounded: if it ever expires nothing is
- *   quantised, *x_scale is set to NaN and the workspace must be zero-filled
- *   again.
- * Requires M > 0, K > 0, K % 8 == 0, X and Xq 16-byte aligned.
+ *   grid-wide barrier.  Its waits are bounded (2 s), and the outcome is all or
+ *   nothing as far as the scale goes: *x_scale is set to NaN when the kernel
+ *   starts and receives the real scale only after EVERY CTA has passed the
+ *   barrier.  If a wait ever expires, the int32 at byte offset
+ *   GPUSQ_QUANT_ACT_STATUS_OFFSET of the workspace becomes GPUSQ_ERR_TIMEOUT
+ *   (it is 0 otherwise), *x_scale stays NaN, Xq is undefined (CTAs that had
+ *   passed the barrier may have written their part), and the workspace must be
+ *   zero-filled again before it is reused.  The host call never waits for the
+ *   device; a caller that wants to know reads the status word (or tests the
+ *   scale) after synchronising.
+ * Requires M > 0, K > 0, K % 8 == 0, X and Xq 16-byte aligned.  The first
+ * GPUSQ_SCALE_COMPUTE call on each device (with that device current) opts the
+ * kernel in to large shared memory; it is safe from several threads.
  */
+#define GPUSQ_QUANT_ACT_STATUS_OFFSET 8196
 size_t gpusq_quant_act_workspace(int64_t M, int K);
 int gpusq_quant_act(const void *X, int8_t *Xq, float *x_scale, int scale_mode, int64_t M, int K,
                     void *workspace, size_t ws_bytes, void *stream);
@@ -219,6 +229,38 @@ int gpusq_spgemm_i8(const int8_t *Xq, const void *Wpacked, const float *w_scale,
                     const float *x_scale, const float *bias, int act, int out_type,
                     const float *out_scale, void *Y, int64_t M, int N, int K, int32_t *status_buf,
                     void *stream);
+
+/* ---------------------------------------------------------------------------
+ * Chaining layers (Sec. 2.2: a quantise node in front of every GEMM and a
+ * de-quantise node behind it, through the whole deployed model; Sec. 4.1:
+ * deployment as INT8 layers).  Two ways to spare the next layer's quantise
+ * node its pass over the tensor for the maximum:
+ *   - gpusq_spgemm_i8 with GPUSQ_OUT_I8 writes the next layer's INT8 codes
+ *     directly (supplied *out_scale, e.g. calibrated); the next
+ *     gpusq_spgemm_i8 reads them with x_scale = that out_scale;
+ *   - gpusq_spgemm_i8_absmax writes FP16 and, beside it, the largest
+ *     magnitude of what it wrote; gpusq_quant_act_absmax then derives the
+ *     per-tensor scale from that number and quantises in ONE pass, with the
+ *     same result as gpusq_quant_act(GPUSQ_SCALE_COMPUTE) on that tensor.
+ *
+ * gpusq_spgemm_i8_absmax: gpusq_spgemm_i8 with GPUSQ_OUT_F16 (same arguments,
+ *   same Y, bit for bit) plus
+ *   y_absmax device float[1]: max over all m < M, n < N of |Y[m,n]| (the
+ *     rounded binary16 values) is MERGED into it (an atomic maximum on the
+ *     bit pattern), so it must hold 0.0f -- or the running maximum of the
+ *     tensors it is to cover -- on entry.  Finite outputs assumed.
+ * gpusq_quant_act_absmax: X [M, K] f16 in, Xq [M, K] i8 out,
+ *   absmax device float[1] in (max |X|), x_scale device float[1] out:
+ *   *x_scale = *absmax / 127 (1.0 when it is 0), codes as gpusq_quant_act.
+ *   absmax and x_scale must be different addresses.  One launch, no workspace.
+ *   Requires M > 0, K % 8 == 0, X / Xq 16-byte aligned.
+ */
+int gpusq_spgemm_i8_absmax(const int8_t *Xq, const void *Wpacked, const float *w_scale,
+                           const float *x_scale, const float *bias, int act, void *Y,
+                           float *y_absmax, int64_t M, int N, int K, int32_t *status_buf,
+                           void *stream);
+int gpusq_quant_act_absmax(const void *X, int8_t *Xq, float *x_scale, const float *absmax,
+                           int64_t M, int K, void *stream);
 
 /* ---------------------------------------------------------------------------
  * The FP16 2:4 sparse model.  Paper: Sec. 3.1 (the compressed FP16 operand:

@@ -5,9 +5,9 @@
  * kernels through every tile height and through mixed tile heights on small
  * shapes; results never depend on them.
  *
- * Both settings are process-wide atomics read by every later gpusq_spgemm_i8 /
- * gpusq_gemm_i8_dense / gpusq_spgemm_f16 call of the process, from any thread;
- * they are meant to be set while no other thread is issuing GEMM calls.
+ * All settings are process-wide atomics read by every later call of the
+ * process, from any thread; they are meant to be set while no other thread is
+ * issuing calls.
  */
 #ifndef GPUSQ_TESTING_H
 #define GPUSQ_TESTING_H
@@ -23,6 +23,14 @@ int gpusq_set_block_tokens(int block_t);
 /* Mixed heights: the first n_big token tiles block_t tokens high (block_t a
  * multiple of 32 in [64, 224]), the rest block_t - 32, as many as cover M. */
 int gpusq_set_tile_mix(int block_t, int n_big);
+
+/* Bound of the device-side waits of gpusq_quant_act's one-launch kernel, in
+ * nanoseconds (default 2 s), and, with withhold_last_cta != 0, a planted
+ * failure made on purpose in an allowed form: the last CTA never publishes its
+ * maximum, so every CTA's bounded wait runs out, the kernel returns, and the
+ * status word and the NaN scale described in gpusq.h can be observed.  Nothing
+ * faults or hangs: the waits end at the bound. */
+int gpusq_set_quant_act_wait(unsigned long long limit_ns, int withhold_last_cta);
 
 #ifdef __cplusplus
 }

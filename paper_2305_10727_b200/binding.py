@@ -24,7 +24,8 @@ SCALE_COMPUTE, SCALE_GIVEN = 0, 1
 EXPORTS = (
     "gpusq_status_string", "gpusq_prune24", "gpusq_quant_weight", "gpusq_compress24",
     "gpusq_decompress24", "gpusq_packed_bytes", "gpusq_pack24", "gpusq_quant_act_workspace",
-    "gpusq_quant_act", "gpusq_quant_act_static", "gpusq_patch_quant", "gpusq_spgemm_i8", "gpusq_gemm_i8_dense", "gpusq_set_block_tokens", "gpusq_set_tile_mix",
+    "gpusq_quant_act", "gpusq_quant_act_static", "gpusq_patch_quant", "gpusq_spgemm_i8", "gpusq_gemm_i8_dense", "gpusq_set_block_tokens", "gpusq_set_tile_mix", "gpusq_set_quant_act_wait",
+    "gpusq_spgemm_i8_absmax", "gpusq_quant_act_absmax",
     "gpusq_compress24_f16", "gpusq_packed_bytes_f16", "gpusq_pack24_f16", "gpusq_spgemm_f16",
 )
 
@@ -65,8 +66,11 @@ def load() -> ctypes.CDLL:
     gemm_args = [vp, vp, vp, vp, vp, i32, i32, vp, vp, i64, i32, i32, vp, vp]
     lib.gpusq_spgemm_i8.argtypes = gemm_args
     lib.gpusq_gemm_i8_dense.argtypes = gemm_args
+    lib.gpusq_spgemm_i8_absmax.argtypes = [vp, vp, vp, vp, vp, i32, vp, vp, i64, i32, i32, vp, vp]
+    lib.gpusq_quant_act_absmax.argtypes = [vp, vp, vp, vp, i64, i32, vp]
     lib.gpusq_set_block_tokens.argtypes = [i32]
     lib.gpusq_set_tile_mix.argtypes = [i32, i32]
+    lib.gpusq_set_quant_act_wait.argtypes = [ctypes.c_ulonglong, i32]
     lib.gpusq_compress24_f16.argtypes = [vp, vp, vp, i32, i32, vp]
     lib.gpusq_packed_bytes_f16.argtypes = [i32, i32]
     lib.gpusq_packed_bytes_f16.restype = sz
@@ -183,6 +187,20 @@ def quant_act(X: torch.Tensor, Xq: Optional[torch.Tensor] = None, x_scale: Optio
     return Xq, x_scale
 
 
+QUANT_ACT_STATUS_OFFSET = 8196       # GPUSQ_QUANT_ACT_STATUS_OFFSET of gpusq.h
+
+
+def quant_act_status(workspace: torch.Tensor) -> int:
+    """The status word gpusq_quant_act keeps in its workspace (0, or 7 = a bounded wait expired).  Synchronises."""
+    word = workspace.view(torch.uint8)[QUANT_ACT_STATUS_OFFSET:QUANT_ACT_STATUS_OFFSET + 4].view(torch.int32)
+    return int(word.cpu().item())
+
+
+def set_quant_act_wait(limit_ns: int, withhold_last_cta: bool = False) -> None:
+    """Test hook (gpusq_testing.h): bound of the one-launch kernel's waits; optionally plant an arrival that never comes."""
+    _check(load().gpusq_set_quant_act_wait(int(limit_ns), 1 if withhold_last_cta else 0), "gpusq_set_quant_act_wait")
+
+
 def quant_act_static(X: torch.Tensor, Xq: Optional[torch.Tensor] = None, x_scale: Optional[torch.Tensor] = None,
                      scale_mode: int = SCALE_COMPUTE):
     """gpusq_quant_act_static: no workspace argument; the library's own fixed scratch is used."""
@@ -251,6 +269,35 @@ def spgemm_i8(Xq: torch.Tensor, Wpacked: torch.Tensor, N: int, w_scale=None, x_s
               act: int = ACT_NONE, out_type: int = OUT_F16, out_scale=None, Y=None, status_buf=None):
     return _gemm("gpusq_spgemm_i8", Xq, Wpacked, w_scale, x_scale, bias, act, out_type, out_scale, Y, N,
                  status_buf)
+
+
+def spgemm_i8_absmax(Xq: torch.Tensor, Wpacked: torch.Tensor, N: int, w_scale, x_scale, bias=None,
+                     act: int = ACT_NONE, Y=None, y_absmax=None, status_buf=None):
+    """gpusq_spgemm_i8_absmax: FP16 output plus max |Y| merged into y_absmax (float32[1], zeroed here if not given)."""
+    _dev(Xq, torch.int8, "Xq")
+    M, K = Xq.shape
+    if Y is None:
+        Y = torch.empty((M, N), dtype=torch.float16, device=Xq.device)
+    if y_absmax is None:
+        y_absmax = torch.zeros((1,), dtype=torch.float32, device=Xq.device)
+    _check(load().gpusq_spgemm_i8_absmax(_ptr(Xq), _ptr(Wpacked), _ptr(w_scale), _ptr(x_scale), _ptr(bias), act,
+                                         _ptr(Y), _ptr(y_absmax), M, N, K, _ptr(status_buf), _stream()),
+           "gpusq_spgemm_i8_absmax")
+    return Y, y_absmax
+
+
+def quant_act_absmax(X: torch.Tensor, absmax: torch.Tensor, Xq: Optional[torch.Tensor] = None,
+                     x_scale: Optional[torch.Tensor] = None):
+    """gpusq_quant_act_absmax: one-pass quantisation with the scale derived from a known max |X|."""
+    _dev(X, torch.float16, "X")
+    M, K = X.shape
+    if Xq is None:
+        Xq = torch.empty((M, K), dtype=torch.int8, device=X.device)
+    if x_scale is None:
+        x_scale = torch.empty((1,), dtype=torch.float32, device=X.device)
+    _check(load().gpusq_quant_act_absmax(_ptr(X), _ptr(Xq), _ptr(x_scale), _ptr(absmax), M, K, _stream()),
+           "gpusq_quant_act_absmax")
+    return Xq, x_scale
 
 
 def gemm_i8_dense(Xq: torch.Tensor, Wq: torch.Tensor, w_scale=None, x_scale=None, bias=None,

@@ -4,6 +4,7 @@
 // per tensor; no shared-memory staging is needed (no reuse across threads).
 #include <cuda_fp16.h>
 
+#include <atomic>
 #include <mutex>
 
 #include "common.cuh"
@@ -312,8 +313,9 @@ pack24_f16_kernel(const uint16_t *__restrict__ vals, const uint8_t *__restrict__
 }
 
 // --------------------------------------------------------------- quant_act
+constexpr int kMaxDevices = 64;
 constexpr int kMaxPartials = 2048;   // workspace: one 32-bit partial maximum per block ...
-constexpr int kWorkspaceExtra = 64;  // ... and, behind them, the words of the grid-wide barrier (8-byte aligned)
+constexpr int kWorkspaceExtra = 64;  // ... and, behind them, the control words of the one-launch kernel
 
 __device__ __forceinline__ uint32_t absmax_bits8(uint4 v)
 {
@@ -362,14 +364,19 @@ __device__ __forceinline__ uint2 quant8_f16(uint4 v, const QuantScale &a)
 }
 
 // n_partials > 0: the scale is derived from the partial maxima and written to
-// *x_scale by block 0; n_partials == 0: *x_scale is read.
+// *x_scale by block 0; absmax != NULL: it is derived from *absmax (the tensor's maximum magnitude,
+// left there by the kernel that produced X) and written; otherwise *x_scale is read.
 __global__ void __launch_bounds__(kThreads)
 act_quant_kernel(const uint4 *__restrict__ X, uint2 *__restrict__ Xq, float *x_scale,
-                 const uint32_t *__restrict__ partial, int n_partials, int64_t vec8)
+                 const uint32_t *__restrict__ partial, int n_partials, int64_t vec8,
+                 const float *__restrict__ absmax = nullptr)
 {
     __shared__ float red[kThreads / 32];
     float s;
-    if (n_partials > 0) {
+    if (absmax) {
+        s = scale_from_amax(__ldg(absmax));
+        if (blockIdx.x == 0 && threadIdx.x == 0) *x_scale = s;
+    } else if (n_partials > 0) {
         uint32_t m = 0;
         for (int i = threadIdx.x; i < n_partials; i += blockDim.x) m = max(m, __ldg(partial + i));
         const uint32_t bits = (uint32_t)block_max((float)m, red);
@@ -507,16 +514,29 @@ patch_quant_kernel(const __half *__restrict__ img, int8_t *__restrict__ Xq, floa
 
 // ---- one-launch activation quantisation (scale computed from the tensor) ----
 // A cooperative grid of one 1024-thread CTA per SM.  Each CTA owns a contiguous slice of X:
-//   1. reads it once from HBM, keeps as much of it as fits in shared memory, finds max|x|;
-//   2. merges its maximum into a global one and crosses a grid-wide barrier (three words in the
-//      workspace, zero before and after every call; the wait is bounded);
+//   1. bulk-asynchronous copies bring as much of the slice as fits into shared memory (sixteen-KB
+//      pieces, each completing on its own mbarrier, all in flight at once); what does not fit is
+//      read with plain loads, last, so that it is still in L2 in step 3.  The threads take the
+//      maximum |x| of every piece as it lands;
+//   2. grid-wide maximum: the CTA merges its maximum into a word of the workspace, counts itself in
+//      and polls, with a bounded wait, until every CTA has been counted;
 //   3. quantises the slice, from shared memory where it was kept, and writes the codes.
-// So X crosses HBM once when a slice fits (up to ~200 KB per SM, 29 MB per tensor) and there is
-// one launch instead of two.  If the barrier wait expires nothing is quantised and *x_scale = NaN.
+// So X crosses HBM once when a slice fits (up to 192 KB per SM, 28 MB per tensor) and there is one
+// launch instead of two.
+// All or nothing: block 0 sets *x_scale to NaN on entry; the CTA that is last to finish step 2 (a
+// counter, off the critical path) writes the real scale and puts the control words back to zero.  A
+// CTA whose wait expires records GPUSQ_ERR_TIMEOUT in the status word and returns without
+// quantising; the scale then stays NaN and the workspace has to be zero-filled again.
 constexpr int kFusedThreads = 1024;
-constexpr int kFusedCacheVecs = 12800;                           // 16-byte vectors kept per CTA (200 KB)
+constexpr int kPieceVecs = 1024;                                 // 16-byte vectors per bulk copy (16 KB): one per thread
+constexpr int kMaxPieces = 12;
+constexpr int kFusedCacheVecs = kPieceVecs * kMaxPieces;         // vectors kept per CTA (192 KB)
 constexpr int kFusedSmemBytes = kFusedCacheVecs * 16;
-constexpr uint64_t kGridWaitLimitNs = 2000000000ull;             // 2 s
+constexpr int kWsDone = kMaxPartials;                            // workspace words: CTAs past the barrier ...
+constexpr int kWsStatus = kMaxPartials + 1;                      // ... status (0 or GPUSQ_ERR_TIMEOUT) ...
+constexpr int kWsBarrier = kMaxPartials + 2;                     // ... and the 8-byte word {arrivals, maximum}
+static std::atomic<unsigned long long> g_grid_wait_ns{2000000000ull};    // bound of the waits below (2 s)
+static std::atomic<int> g_withhold_slot{0};                      // test hook: the last CTA does not publish
 
 __device__ __forceinline__ uint64_t globaltimer_now()
 {
@@ -525,45 +545,70 @@ __device__ __forceinline__ uint64_t globaltimer_now()
     return t;
 }
 
+__device__ __forceinline__ bool mbar_try_wait_parity0(uint32_t bar)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred P;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 P, [%1], 0, 1000;\n"
+        "selp.u32 %0, 1, 0, P;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(bar)
+        : "memory");
+    return ok != 0;
+}
+
 __global__ void __launch_bounds__(kFusedThreads, 1)
 act_quant_fused_kernel(const uint4 *__restrict__ X, uint2 *__restrict__ Xq, float *x_scale,
-                       uint32_t *counters, int64_t vec8)
+                       uint32_t *ws, int64_t vec8, unsigned long long wait_ns, int withhold)
 {
-    extern __shared__ uint4 cache[];
+    extern __shared__ __align__(128) uint4 cache[];
     __shared__ float red[kFusedThreads / 32];
-    __shared__ uint32_t barrier_ok, grid_max_bits;
+    __shared__ __align__(8) uint64_t piece_bar[kMaxPieces];
+    __shared__ uint32_t gave_up;
     const int64_t per = (vec8 + gridDim.x - 1) / gridDim.x;
     const int64_t lo = (int64_t)blockIdx.x * per;
     const int64_t hi = lo + per < vec8 ? lo + per : vec8;
     const int tid = threadIdx.x;
-    // the next kernel of the stream may be scheduled as soon as CTAs of this grid make room
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     // The slice in 32-bit terms: n vectors from Xs; the first n_kept of them stay in shared memory.
     const int n = hi > lo ? (int)(hi - lo) : 0;             // host side: per < 2^31
     const int n_kept = n < kFusedCacheVecs ? n : kFusedCacheVecs;
+    const int pieces = (n_kept + kPieceVecs - 1) / kPieceVecs;
     const uint4 *Xs = X + lo;
     uint2 *Xqs = Xq + lo;
 
-    // 1. maximum of the slice
-    uint32_t m = 0;
-    int i = tid;
-    for (; i + 3 * kFusedThreads < n_kept; i += 4 * kFusedThreads) {
-        uint4 v[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) v[u] = __ldcs(Xs + i + u * kFusedThreads);   // kept: not needed from L2 again
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            m = max(m, absmax_bits8(v[u]));
-            cache[i + u * kFusedThreads] = v[u];
+    if (tid == 0) {
+        for (int c = 0; c < pieces; ++c)
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"((uint32_t)__cvta_generic_to_shared(&piece_bar[c])));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        gave_up = 0;
+    }
+    __syncthreads();
+    // the previous kernel of the stream (a producer of X, or a user of the workspace) is complete from here on
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    // the next kernel of the stream may be scheduled as soon as CTAs of this grid make room
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (blockIdx.x == 0 && tid == 0) *x_scale = __int_as_float(0x7FC00000);
+
+    // 1. the slice into shared memory, all pieces in flight at once
+    if (tid == 0) {
+        for (int c = 0; c < pieces; ++c) {
+            const int v0 = c * kPieceVecs;
+            const uint32_t bytes = (uint32_t)((n_kept - v0 < kPieceVecs ? n_kept - v0 : kPieceVecs) * 16);
+            const uint32_t bar = (uint32_t)__cvta_generic_to_shared(&piece_bar[c]);
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                             (uint32_t)__cvta_generic_to_shared(cache + v0)),
+                         "l"(Xs + v0), "r"(bytes), "r"(bar)
+                         : "memory");
         }
     }
-    for (; i < n_kept; i += kFusedThreads) {
-        const uint4 v = __ldcs(Xs + i);
-        m = max(m, absmax_bits8(v));
-        cache[i] = v;
-    }
-    // the rest is re-read in step 3: plain loads leave it in L2 (i continues at n_kept + its lane offset)
+    // what does not fit: maximum only, plain loads that leave the lines in L2 for step 3
+    uint32_t m = 0;
+    int i = n_kept + tid;
     for (; i + 3 * kFusedThreads < n; i += 4 * kFusedThreads) {
         uint4 v[4];
 #pragma unroll
@@ -572,49 +617,82 @@ act_quant_fused_kernel(const uint4 *__restrict__ X, uint2 *__restrict__ Xq, floa
         for (int u = 0; u < 4; ++u) m = max(m, absmax_bits8(v[u]));
     }
     for (; i < n; i += kFusedThreads) m = max(m, absmax_bits8(__ldg(Xs + i)));
-    const uint32_t mine = (uint32_t)block_max((float)m, red);
-
-    // 2. grid-wide maximum.  One 8-byte word holds {arrivals, maximum}: a CTA first merges its maximum,
-    // then counts itself in, so a single 8-byte read that sees every arrival also sees the final
-    // maximum.  counters[2] counts the CTAs that have read it; the last of them puts all three words
-    // back to zero, the state the next call on this workspace expects.
-    if (tid == 0) {
-        atomicMax(counters + 1, mine);
-        __threadfence();
-        atomicAdd(counters, 1u);
-        const uint64_t t0 = globaltimer_now();
-        uint32_t ok = 1;
-        uint2 word;
-        for (uint32_t it = 1;; ++it) {
-            word = __ldcv(reinterpret_cast<const uint2 *>(counters));
-            if (word.x >= gridDim.x) break;
-            if ((it & 255u) == 0u && globaltimer_now() - t0 > kGridWaitLimitNs) {
-                ok = 0;
+    // the pieces as they land: thread t looks at vector t of each
+    const uint64_t t0 = globaltimer_now();
+    bool ok = true;
+    for (int c = 0; c < pieces && ok; ++c) {
+        const uint32_t bar = (uint32_t)__cvta_generic_to_shared(&piece_bar[c]);
+        while (!mbar_try_wait_parity0(bar)) {
+            if (globaltimer_now() - t0 > wait_ns) {
+                ok = false;
                 break;
             }
         }
-        if (ok && atomicAdd(counters + 2, 1u) == gridDim.x - 1) {
-            __stcg(reinterpret_cast<uint2 *>(counters), make_uint2(0u, 0u));
-            counters[2] = 0;
-        }
-        barrier_ok = ok;
-        grid_max_bits = word.y;
+        const int v = c * kPieceVecs + tid;
+        if (ok && v < n_kept) m = max(m, absmax_bits8(cache[v]));
     }
-    __syncthreads();
-    if (!barrier_ok) {
-        if (blockIdx.x == 0 && tid == 0) *x_scale = __int_as_float(0x7FC00000);
+    if (!ok) gave_up = 1;                                    // benign race: every writer writes 1
+    const uint32_t mine = (uint32_t)block_max((float)m, red);            // has the block-wide barriers
+
+    // 2. grid-wide maximum.  One 8-byte word holds {arrivals, maximum}: a CTA first merges its maximum,
+    // then counts itself in, so a single 8-byte read that sees every arrival also sees the final
+    // maximum; each CTA has one poll in flight at a time, all on one line.
+    uint32_t *bar_word = ws + kWsBarrier;
+    uint32_t seen = 0;
+    if (tid == 0 && !gave_up) {
+        if (!(withhold && blockIdx.x == gridDim.x - 1)) {
+            atomicMax(bar_word + 1, mine);
+            __threadfence();
+            atomicAdd(bar_word, 1u);
+        }
+        for (uint32_t it = 1;; ++it) {
+            const uint2 word = __ldcv(reinterpret_cast<const uint2 *>(bar_word));
+            if (word.x >= gridDim.x) {
+                seen = word.y;
+                break;
+            }
+            if ((it & 63u) == 0u && globaltimer_now() - t0 > wait_ns) {
+                gave_up = 1;
+                break;
+            }
+        }
+    }
+    const uint32_t all = (uint32_t)block_max((float)seen, red);
+    if (gave_up) {
+        if (tid == 0) atomicExch(ws + kWsStatus, (uint32_t)GPUSQ_ERR_TIMEOUT);
+        // bulk copies that may still be in flight write into this CTA's shared memory: wait for them (bounded)
+        if (tid == 0) {
+            const uint64_t t1 = globaltimer_now();
+            for (int c = 0; c < pieces; ++c) {
+                const uint32_t bar = (uint32_t)__cvta_generic_to_shared(&piece_bar[c]);
+                while (!mbar_try_wait_parity0(bar) && globaltimer_now() - t1 < wait_ns) {
+                }
+            }
+        }
+        __syncthreads();
         return;
     }
-    const float s = scale_from_amax(__half2float(__ushort_as_half((unsigned short)grid_max_bits)));
-    if (blockIdx.x == 0 && tid == 0) *x_scale = s;
+    if (tid == 0) {
+        // the last CTA past the barrier: nobody polls any more, so the workspace goes back to zero and
+        // the scale, which tells the caller that every CTA came through, is written
+        __threadfence();
+        if (atomicAdd(ws + kWsDone, 1u) == gridDim.x - 1) {
+            __stcg(reinterpret_cast<uint2 *>(bar_word), make_uint2(0u, 0u));
+            __stcg(ws + kWsDone, 0u);
+            *x_scale = scale_from_amax(__half2float(__ushort_as_half((unsigned short)all)));
+        }
+    }
+    const float s = scale_from_amax(__half2float(__ushort_as_half((unsigned short)all)));
     const QuantScale a = make_quant_scale(s);
 
     // 3. quantise the slice: what was kept, from shared memory; the rest, from L2 / HBM
     for (i = tid; i < n_kept; i += kFusedThreads) __stcs(Xqs + i, quant8_f16<false>(cache[i], a));
-    for (; i + kFusedThreads < n; i += 2 * kFusedThreads) {
-        const uint4 v0 = __ldg(Xs + i), v1 = __ldg(Xs + i + kFusedThreads);
-        __stcs(Xqs + i, quant8_f16<false>(v0, a));
-        __stcs(Xqs + i + kFusedThreads, quant8_f16<false>(v1, a));
+    for (; i + 3 * kFusedThreads < n; i += 4 * kFusedThreads) {
+        uint4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) v[u] = __ldg(Xs + i + u * kFusedThreads);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) __stcs(Xqs + i + u * kFusedThreads, quant8_f16<false>(v[u], a));
     }
     for (; i < n; i += kFusedThreads) __stcs(Xqs + i, quant8_f16<false>(__ldg(Xs + i), a));
 }
@@ -625,7 +703,6 @@ act_quant_fused_kernel(const uint4 *__restrict__ X, uint2 *__restrict__ Xq, floa
 // looked up once per device with that device current.
 constexpr int64_t kStaticMaxElems = (int64_t)1 << 32;     // largest M*K the static entry point accepts
 static __device__ __align__(256) uint32_t g_act_scratch[kMaxPartials];
-constexpr int kMaxDevices = 64;
 static std::mutex g_scratch_mutex;
 static uint32_t *g_scratch_addr[kMaxDevices] = {};
 
@@ -772,6 +849,7 @@ size_t gpusq_quant_act_workspace(int64_t M, int K)
 int gpusq_quant_act(const void *X, int8_t *Xq, float *x_scale, int scale_mode, int64_t M, int K,
                     void *workspace, size_t ws_bytes, void *stream)
 {
+    static_assert(GPUSQ_QUANT_ACT_STATUS_OFFSET == kWsStatus * sizeof(uint32_t), "status word as documented");
     if (!X || !Xq || !x_scale) return GPUSQ_ERR_NULL;
     if (M <= 0 || K <= 0 || K % 8) return GPUSQ_ERR_SHAPE;
     if (scale_mode != GPUSQ_SCALE_COMPUTE && scale_mode != GPUSQ_SCALE_GIVEN) return GPUSQ_ERR_ARG;
@@ -784,31 +862,45 @@ int gpusq_quant_act(const void *X, int8_t *Xq, float *x_scale, int scale_mode, i
     const int64_t vec8 = M * (int64_t)K / 8;
     cudaStream_t s = (cudaStream_t)stream;
     if (scale_mode == GPUSQ_SCALE_COMPUTE) {
-        // one cooperative launch: every CTA must be resident for the grid-wide barrier
-        static std::once_flag once;
-        static cudaError_t attr_err = cudaSuccess;
-        std::call_once(once, [] {
-            attr_err = cudaFuncSetAttribute(act_quant_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                            kFusedSmemBytes);
-        });
-        if (attr_err != cudaSuccess) return GPUSQ_ERR_CUDA;
-        int per_sm = 0;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, act_quant_fused_kernel, kFusedThreads,
-                                                          kFusedSmemBytes) != cudaSuccess || per_sm < 1)
-            return GPUSQ_ERR_CUDA;
+        // one cooperative launch: every CTA must be resident for the grid-wide barrier.  The opt-in to
+        // large dynamic shared memory is per device.
+        static std::mutex mu;
+        static uint8_t attr_state[kMaxDevices] = {};          // 1 = set, 2 = failed
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return GPUSQ_ERR_CUDA;
+        {
+            std::lock_guard<std::mutex> lock(mu);
+            if (attr_state[dev] == 0) {
+                const bool ok = cudaFuncSetAttribute(act_quant_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                     kFusedSmemBytes) == cudaSuccess;
+                if (!ok) (void)cudaGetLastError();
+                attr_state[dev] = ok ? 1 : 2;
+            }
+            if (attr_state[dev] != 1) return GPUSQ_ERR_CUDA;
+        }
         int grid = num_sms();
         if (grid > kMaxPartials) grid = kMaxPartials;
         // small tensors: no more CTAs than give every thread two vectors (fewer arrivals at the barrier)
         const int64_t want = ceil_div(vec8, 2 * kFusedThreads);
         if ((int64_t)grid > want) grid = (int)(want < 1 ? 1 : want);
         if (ceil_div(vec8, grid) > 0x7FFFFFFF) return GPUSQ_ERR_SHAPE;      // a CTA's slice is indexed with 32 bits
-        uint32_t *counters = reinterpret_cast<uint32_t *>(workspace) + kMaxPartials;
-        const uint4 *Xv = reinterpret_cast<const uint4 *>(X);
-        uint2 *Xqv = reinterpret_cast<uint2 *>(Xq);
-        int64_t n = vec8;
-        void *args[] = {&Xv, &Xqv, &x_scale, &counters, &n};
-        if (cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(act_quant_fused_kernel), dim3(grid),
-                                        dim3(kFusedThreads), args, kFusedSmemBytes, s) != cudaSuccess) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)grid, 1, 1);
+        cfg.blockDim = dim3(kFusedThreads, 1, 1);
+        cfg.dynamicSmemBytes = kFusedSmemBytes;
+        cfg.stream = s;
+        cudaLaunchAttribute attr[2];
+        attr[0].id = cudaLaunchAttributeCooperative;
+        attr[0].val.cooperative = 1;
+        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;     // set up while the previous kernel drains
+        attr[1].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 2;
+        const unsigned long long wait_ns = g_grid_wait_ns.load(std::memory_order_relaxed);
+        const int withhold = g_withhold_slot.load(std::memory_order_relaxed);
+        if (cudaLaunchKernelEx(&cfg, act_quant_fused_kernel, reinterpret_cast<const uint4 *>(X),
+                               reinterpret_cast<uint2 *>(Xq), x_scale, reinterpret_cast<uint32_t *>(workspace), vec8,
+                               wait_ns, withhold) != cudaSuccess) {
             (void)cudaGetLastError();
             return GPUSQ_ERR_CUDA;
         }
@@ -817,6 +909,28 @@ int gpusq_quant_act(const void *X, int8_t *Xq, float *x_scale, int scale_mode, i
     act_quant_kernel<<<grid_for(ceil_div(vec8, 2), 8), kThreads, 0, s>>>(
         reinterpret_cast<const uint4 *>(X), reinterpret_cast<uint2 *>(Xq), x_scale, nullptr, 0, vec8);
     return launch_status();
+}
+
+int gpusq_quant_act_absmax(const void *X, int8_t *Xq, float *x_scale, const float *absmax, int64_t M, int K,
+                           void *stream)
+{
+    if (!X || !Xq || !x_scale || !absmax) return GPUSQ_ERR_NULL;
+    if (M <= 0 || K <= 0 || K % 8) return GPUSQ_ERR_SHAPE;
+    if (x_scale == absmax) return GPUSQ_ERR_ARG;
+    if (!aligned(X, 16) || !aligned(Xq, 16)) return GPUSQ_ERR_ALIGN;
+    if (int st = check_arch()) return st;
+    const int64_t vec8 = M * (int64_t)K / 8;
+    act_quant_kernel<<<grid_for(ceil_div(vec8, 2), 8), kThreads, 0, (cudaStream_t)stream>>>(
+        reinterpret_cast<const uint4 *>(X), reinterpret_cast<uint2 *>(Xq), x_scale, nullptr, 0, vec8, absmax);
+    return launch_status();
+}
+
+int gpusq_set_quant_act_wait(unsigned long long limit_ns, int withhold_last_cta)
+{
+    if (limit_ns == 0) return GPUSQ_ERR_ARG;
+    g_grid_wait_ns.store(limit_ns, std::memory_order_relaxed);
+    g_withhold_slot.store(withhold_last_cta ? 1 : 0, std::memory_order_relaxed);
+    return GPUSQ_OK;
 }
 
 int gpusq_quant_act_static(const void *X, int8_t *Xq, float *x_scale, int scale_mode, int64_t M, int K,

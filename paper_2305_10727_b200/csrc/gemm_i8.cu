@@ -111,6 +111,7 @@ struct GemmParams {
     const float *bias;
     const float *out_scale;
     void *Y;
+    float *y_absmax;  // FP16 output only, nullable: max |Y| over the rounded outputs is merged into it
     int32_t *status;
     int64_t M;
     int N;
@@ -248,6 +249,7 @@ struct EpiF16 {
     uint32_t buf_addr, full_bar, free_bar, buf_idx, free_parity;
     uint32_t stm_off;          // this lane's stmatrix row address inside a staging tile (second one: + 2048)
     float2 sc2[2], bi2[2];     // scale and bias of this thread's two features, duplicated for packed math
+    float amax;                // kAmax: largest |y| this thread has produced for a token that exists
 
     __device__ __forceinline__ void release(int acc)
     {
@@ -258,9 +260,11 @@ struct EpiF16 {
 
     // One chunk held in v (its load was issued earlier).  next_taddr != 0: issue this warp's next
     // load into vn; otherwise v was the warp's last chunk of the tile and the accumulator is released.
-    template <bool kGelu>
+    // rows: tokens of the chunk that exist (32 except at the end of the tensor); only kAmax looks at
+    // it, the stores clip by themselves.
+    template <bool kGelu, bool kAmax>
     __device__ __forceinline__ bool step(uint32_t (&v)[16], uint32_t (&vn)[16], uint32_t next_taddr, int acc,
-                                         int tile)
+                                         int tile, int rows)
     {
         ptx::tmem_ld_wait_regs(v);
         if (next_taddr)
@@ -280,6 +284,17 @@ struct EpiF16 {
                 if (kGelu) y = gelu_pair(y);
                 const __half2 hh = __floats2half2_rn(y.x, y.y);   // low = token 2(t%4), high = +1
                 pk[2 * i + j] = *reinterpret_cast<const uint32_t *>(&hh);
+                if (kAmax) {
+                    // rounding is monotonic: the maximum of the rounded outputs is the rounded maximum.
+                    // Rows past the end of the tensor hold the bias only and do not count.
+                    const int tok = 8 * i + 2 * (lane & 3);
+                    if (rows >= kChunkT) {
+                        amax = fmaxf(amax, fmaxf(fabsf(y.x), fabsf(y.y)));
+                    } else {
+                        if (tok < rows) amax = fmaxf(amax, fabsf(y.x));
+                        if (tok + 1 < rows) amax = fmaxf(amax, fabsf(y.y));
+                    }
+                }
             }
         // the staging tile's previous contents have been stored
         bool to;
@@ -307,13 +322,14 @@ struct EpiF16 {
         return true;
     }
 
-    template <bool kGelu>
+    template <bool kGelu, bool kAmax>
     __device__ __forceinline__ void run()
     {
         const int quarter = warp & 3;                      // tensor-memory lanes [32q, 32q+32) are this warp's to read
         const int half = ((warp - 2) >> 2) & 1;            // which 16 of them
         const int par = (warp - 2) >> 3;                   // which chunks: every other one
         const int nofs = quarter * 32 + 16 * half + (lane >> 2);       // this thread's first feature in the CTA's 128
+        amax = 0.0f;
         {
             // stmatrix row of this lane: token 8 (mid / 2) + r of the tile, 16-byte column c16 (128-byte swizzle)
             const int mid = lane >> 3, r = lane & 7;
@@ -385,24 +401,40 @@ struct EpiF16 {
                              (uint32_t)(acc * kAccStride + c0 * kChunkT);
             uint32_t v0[16], v1[16];
             ptx::tmem_ld_16x256b_x4(taddr, v0);
+            // tokens that exist from this warp's chunk on (at least 32 everywhere but at the end of the tensor)
+            const int64_t ahead = M - m0 - (int64_t)c0 * kChunkT;
+            int rows = ahead > 4 * kMaxBlockT ? 4 * kMaxBlockT : (int)ahead;
             for (;;) {
                 taddr += 2 * kChunkT;
-                if (!step<kGelu>(v0, v1, --mine ? taddr : 0u, acc, tile)) return;
+                if (!step<kGelu, kAmax>(v0, v1, --mine ? taddr : 0u, acc, tile, rows)) return;
                 if (!mine) break;
+                rows -= 2 * kChunkT;
                 taddr += 2 * kChunkT;
-                if (!step<kGelu>(v1, v0, --mine ? taddr : 0u, acc, tile)) return;
+                if (!step<kGelu, kAmax>(v1, v0, --mine ? taddr : 0u, acc, tile, rows)) return;
                 if (!mine) break;
+                rows -= 2 * kChunkT;
             }
+        }
+        if (kAmax) {
+            // largest |Y| of this warp as the binary16 value that was stored, merged as a bit pattern
+            // (non-negative binary32 values order like their patterns)
+            float m = __half2float(__float2half_rn(amax));
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+            if (lane == 0 && m > 0.0f) atomicMax(reinterpret_cast<unsigned int *>(p->y_absmax), __float_as_uint(m));
         }
     }
 };
 
-// INT8 epilogue of one worker warp (requantised output).  The warp owns the 32 tensor-memory lanes
-// (features) of its quarter and every fourth 32-token chunk; tcgen05.ld in the 32x32b shape gives each
-// thread one feature and consecutive tokens.  Four tokens of a feature are quantised and packed into a
-// word; two shuffle + byte-permute steps transpose 4 x 4 bytes among four neighbouring lanes, so that
-// each lane holds four neighbouring features of one token and writes them with one 4-byte store into
-// a 128-byte-swizzled [32 tokens][128 features] staging tile that the four quarters' warps share.
+// INT8 epilogue of one worker warp (requantised output): the FP16 epilogue's structure with bytes.
+// The warp owns 16 tensor-memory lanes (features) and every other 32-token chunk; tcgen05.ld in the
+// 16x256b shape gives a thread, per block of eight tokens, two neighbouring tokens of features f and
+// f + 8.  Their four codes, packed into one word, are exactly the fragment of the 8-bit matrix store
+// (stmatrix m16n8 b8, transposed): one instruction per chunk writes the warp's 32 tokens x 16 features
+// as 16-byte row pieces into a 128-byte-swizzled [32 tokens][128 features] staging tile that the
+// eight warps of the same chunk parity fill together; a TMA store writes full 128-byte rows of Y.
+constexpr int kI8Bufs = kEpiGroups * kEpiBufs / 2;      // staging tiles per chunk parity (the same shared memory, two rings)
+
 template <bool kTwin>
 struct EpiI8 {
     const GemmParams *p;
@@ -412,6 +444,11 @@ struct EpiI8 {
     float x_scale, out_scale;
     int warp, lane, rank, cluster_id, num_clusters, tiles_n, num_tiles;
 
+    uint32_t buf_addr, full_bar, free_bar, buf_idx, free_parity, ring0, full0, free0;
+    uint32_t stm_off;
+    float2 sc2[2], bi2[2];
+    QuantScale qs;
+
     __device__ __forceinline__ void release(int acc)
     {
         ptx::tc_fence_before();
@@ -420,33 +457,92 @@ struct EpiI8 {
     }
 
     template <bool kGelu>
+    __device__ __forceinline__ bool step(uint32_t (&v)[16], uint32_t (&vn)[16], uint32_t next_taddr, int acc, int tile)
+    {
+        ptx::tmem_ld_wait_regs(v);
+        if (next_taddr)
+            ptx::tmem_ld_16x256b_x4(next_taddr, vn);
+        else
+            release(acc);
+        uint32_t pk[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            // feature f: tokens 8i + 2(t%4), +1; feature f + 8: the same tokens
+            float2 ya = __ffma2_rn(make_float2(__int2float_rn((int32_t)v[4 * i]), __int2float_rn((int32_t)v[4 * i + 1])), sc2[0], bi2[0]);
+            float2 yb = __ffma2_rn(make_float2(__int2float_rn((int32_t)v[4 * i + 2]), __int2float_rn((int32_t)v[4 * i + 3])), sc2[1], bi2[1]);
+            if (kGelu) {
+                ya = gelu_pair(ya);
+                yb = gelu_pair(yb);
+            }
+            // values beyond +-127 out_scale saturate: rare, so they are only detected here (one
+            // compare per four values) and handled, clamp included, by the exact branch
+            const bool beyond = fmaxf(fmaxf(fabsf(ya.x), fabsf(ya.y)), fmaxf(fabsf(yb.x), fabsf(yb.y))) > qs.x_max;
+            uint32_t differ = 0;
+            float2 ma = quant2_sums<false>(ya, qs, differ), mb = quant2_sums<false>(yb, qs, differ);
+            if (differ != 0u || beyond || qs.always_divide) {
+                ma = quant2_exact<true>(ya, qs);
+                mb = quant2_exact<true>(yb, qs);
+            }
+            pk[i] = pack4_low_bytes(ma, mb);
+        }
+        bool to;
+        if (!ptx::mbar_wait_bounded(free_bar, free_parity, &ctl->abort_flag, to)) {
+            if (to && lane == 0) report_timeout(*p, ctl, tile, 2, 200 + (int)buf_idx);
+            return false;
+        }
+        ptx::stmatrix_x4_trans_b8(buf_addr + stm_off, pk[0], pk[1], pk[2], pk[3]);
+        ptx::fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(full_bar);
+        if (++buf_idx == (uint32_t)kI8Bufs) {
+            buf_idx = 0;
+            free_parity ^= 1u;
+            buf_addr = ring0;
+            full_bar = full0;
+            free_bar = free0;
+        } else {
+            buf_addr += kEpiBufBytes;
+            full_bar += 8;
+            free_bar += 8;
+        }
+        return true;
+    }
+
+    template <bool kGelu>
     __device__ __forceinline__ void run()
     {
-        const int quarter = warp & 3;
-        const int sub = (warp - 2) >> 2;                   // 0..3: which chunks, and which staging ring
-        const int g = lane >> 2, l = lane & 3;
-        const uint32_t sel1 = (l & 1) ? 0x3715u : 0x6240u, sel2 = (l & 2) ? 0x3276u : 0x5410u;
-        // this lane's 4 bytes inside a staging row: features 32 q + 4 g .. + 3
-        const int c16 = 2 * quarter + (g >> 2), within = 4 * (g & 3);
-        const uint32_t row_off0 = (uint32_t)(l * 128 + ((c16 ^ l) << 4) + within);
-        const uint32_t row_off1 = (uint32_t)(l * 128 + ((c16 ^ (4 + l)) << 4) + within);
-        const uint32_t ring0 = ptx::smem_u32(epi_smem + sub * kEpiBufs * kEpiBufBytes);
-        const uint32_t full0 = ptx::smem_u32(&ctl->stg_full[sub][0]), free0 = ptx::smem_u32(&ctl->stg_free[sub][0]);
-        uint32_t buf_addr = ring0, full_bar = full0, free_bar = free0, buf_idx = 0, free_parity = 1;
+        const int quarter = warp & 3;                      // tensor-memory lanes [32q, 32q+32) are this warp's to read
+        const int half = ((warp - 2) >> 2) & 1;            // which 16 of them
+        const int par = (warp - 2) >> 3;                   // which chunks: every other one
+        const int nofs = quarter * 32 + 16 * half + (lane >> 2);
+        // this lane's address in the matrix store: row = token `lane` of the chunk, the warp's 16-byte column
+        stm_off = (uint32_t)(lane * 128 + (((2 * quarter + half) ^ (lane & 7)) << 4));
+        // the barriers of the staging tiles, taken as one array: ring `par` uses entries par * kI8Bufs ...
+        ring0 = ptx::smem_u32(epi_smem + par * kI8Bufs * kEpiBufBytes);
+        full0 = ptx::smem_u32(&ctl->stg_full[0][0]) + (uint32_t)(par * kI8Bufs * 8);
+        free0 = ptx::smem_u32(&ctl->stg_free[0][0]) + (uint32_t)(par * kI8Bufs * 8);
+        buf_addr = ring0;
+        full_bar = full0;
+        free_bar = free0;
+        buf_idx = 0;
+        free_parity = 1;                                   // first round: the tiles are free
         const int64_t M = p->M;
         const int N = p->N;
         const float *w_scale = p->w_scale, *bias = p->bias;
-        const QuantScale qs = make_quant_scale(out_scale);
+        qs = make_quant_scale(out_scale);
 
-        float ws_next, bi_next;
+        float ws_next[2], bi_next[2];
         auto fetch = [&](const TileWalk<kTwin> &w) {
             int n0, unused_h;
             int64_t unused;
             w.origin(*p, rank, n0, unused, unused_h);
-            const int n = n0 + quarter * 32 + lane;
-            const bool in = w.tile < num_tiles && n < N;
-            ws_next = in ? __ldg(w_scale + n) : 0.0f;
-            bi_next = (in && bias) ? __ldg(bias + n) : 0.0f;
+            const bool in = w.tile < num_tiles && n0 < N;
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                const int n = n0 + nofs + 8 * j;
+                ws_next[j] = (in && n < N) ? __ldg(w_scale + n) : 0.0f;
+                bi_next[j] = (in && n < N && bias) ? __ldg(bias + n) : 0.0f;
+            }
         };
         TileWalk<kTwin> walk(*p, cluster_id, num_clusters);
         fetch(walk);
@@ -460,8 +556,12 @@ struct EpiI8 {
             const int acc = local & 1;
             const uint32_t acc_phase = (uint32_t)(local >> 1) & 1u;
             const bool n_valid = n0 < N;
-            const float sc = __fmul_rn(ws_next, x_scale);
-            const float2 sc2 = make_float2(sc, sc), bi2 = make_float2(bi_next, bi_next);
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                const float sc = __fmul_rn(ws_next[j], x_scale);
+                sc2[j] = make_float2(sc, sc);
+                bi2[j] = make_float2(bi_next[j], bi_next[j]);
+            }
             fetch(walk);
             bool to;
             if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->tmem_full[acc]), acc_phase, &ctl->abort_flag, to)) {
@@ -474,67 +574,23 @@ struct EpiI8 {
                 const int64_t left = M - m0;
                 nchunks = left >= h ? h / kChunkT : (int)((left + kChunkT - 1) / kChunkT);
             }
-            const int c0 = (sub - local) & 3;              // chunk c belongs to the warps with sub == (c + local) % 4
-            if (c0 >= nchunks) {
+            const int c0 = (par + local) & 1;
+            int mine = (nchunks - c0 + 1) >> 1;
+            if (mine <= 0) {
                 release(acc);
                 continue;
             }
-            const uint32_t tbase = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * kAccStride);
-            for (int c = c0; c < nchunks; c += 4) {
-                uint32_t va[16], vb[16];
-                ptx::tmem_ld_32x32b_x16(tbase + (uint32_t)(c * kChunkT), va);
-                ptx::tmem_ld_32x32b_x16(tbase + (uint32_t)(c * kChunkT + 16), vb);
-                ptx::tmem_ld_wait_regs(va);
-                ptx::tmem_ld_wait_regs(vb);
-                if (c + 4 >= nchunks) release(acc);        // all this warp reads of the tile is in registers
-                if (!ptx::mbar_wait_bounded(free_bar, free_parity, &ctl->abort_flag, to)) {
-                    if (to && lane == 0) report_timeout(*p, ctl, tile, 2, 200 + (int)buf_idx);
-                    return;
-                }
-#pragma unroll
-                for (int w = 0; w < 8; ++w) {
-                    // tokens 4w .. 4w+3 of the chunk, this thread's feature
-                    const uint32_t a0 = w < 4 ? va[4 * w] : vb[4 * w - 16], a1 = w < 4 ? va[4 * w + 1] : vb[4 * w - 15];
-                    const uint32_t a2 = w < 4 ? va[4 * w + 2] : vb[4 * w - 14], a3 = w < 4 ? va[4 * w + 3] : vb[4 * w - 13];
-                    float2 y01 = __ffma2_rn(make_float2(__int2float_rn((int32_t)a0), __int2float_rn((int32_t)a1)), sc2, bi2);
-                    float2 y23 = __ffma2_rn(make_float2(__int2float_rn((int32_t)a2), __int2float_rn((int32_t)a3)), sc2, bi2);
-                    if (kGelu) {
-                        y01 = gelu_pair(y01);
-                        y23 = gelu_pair(y23);
-                    }
-                    // values beyond +-127 out_scale saturate: rare, so they are only detected here (one
-                    // compare per four values) and handled, clamp included, by the exact branch
-                    const bool beyond = fmaxf(fmaxf(fabsf(y01.x), fabsf(y01.y)), fmaxf(fabsf(y23.x), fabsf(y23.y))) > qs.x_max;
-                    uint32_t differ = 0;
-                    float2 m01 = quant2_sums<false>(y01, qs, differ), m23 = quant2_sums<false>(y23, qs, differ);
-                    if (differ != 0u || beyond || qs.always_divide) {
-                        m01 = quant2_exact<true>(y01, qs);
-                        m23 = quant2_exact<true>(y23, qs);
-                    }
-                    const uint32_t word = pack4_low_bytes(m01, m23);          // byte j: token 4w + j
-                    // 4 x 4 byte transpose over lanes 4g .. 4g+3 (features) x tokens 4w .. 4w+3
-                    const uint32_t r1 = __shfl_xor_sync(0xffffffffu, word, 1);
-                    const uint32_t half2tok = __byte_perm(word, r1, sel1);   // two features x two tokens
-                    const uint32_t r2 = __shfl_xor_sync(0xffffffffu, half2tok, 2);
-                    const uint32_t out = __byte_perm(half2tok, r2, sel2);     // features 4g..4g+3 of token 4w + l
-                    // row 4w + l of the tile; (4w + l) & 7 = l or 4 + l, so two offsets serve all eight words
-                    const uint32_t addr = buf_addr + ((w & 1) ? row_off1 : row_off0) + (uint32_t)(w * 512);
-                    asm volatile("st.shared.b32 [%0], %1;" ::"r"(addr), "r"(out) : "memory");
-                }
-                ptx::fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(full_bar);
-                if (++buf_idx == (uint32_t)kEpiBufs) {
-                    buf_idx = 0;
-                    free_parity ^= 1u;
-                    buf_addr = ring0;
-                    full_bar = full0;
-                    free_bar = free0;
-                } else {
-                    buf_addr += kEpiBufBytes;
-                    full_bar += 8;
-                    free_bar += 8;
-                }
+            uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32 + half * 16) << 16) +
+                             (uint32_t)(acc * kAccStride + c0 * kChunkT);
+            uint32_t v0[16], v1[16];
+            ptx::tmem_ld_16x256b_x4(taddr, v0);
+            for (;;) {
+                taddr += 2 * kChunkT;
+                if (!step<kGelu>(v0, v1, --mine ? taddr : 0u, acc, tile)) return;
+                if (!mine) break;
+                taddr += 2 * kChunkT;
+                if (!step<kGelu>(v1, v0, --mine ? taddr : 0u, acc, tile)) return;
+                if (!mine) break;
             }
         }
     }
@@ -542,7 +598,9 @@ struct EpiI8 {
 
 // kOut = GPUSQ_OUT_F16 / _I8 / _I32: one instantiation per output type, so that each epilogue gets its
 // own register allocation
-template <bool kSparse, int kOut, bool kHalf = false, bool kTwin = false>
+// kAmax: the FP16 epilogue also merges max |Y| into a device word (its own instantiation, so that the
+// ordinary kernel's register allocation is untouched)
+template <bool kSparse, int kOut, bool kHalf = false, bool kTwin = false, bool kAmax = false>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kNumThreads, 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_b2, const __grid_constant__ CUtensorMap map_e,
@@ -582,7 +640,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         ptx::mbar_init(ptx::smem_u32(&ctl->drain), 1);
         for (int g = 0; g < kEpiGroups; ++g)
             for (int b = 0; b < gpusq::kEpiBufs; ++b) {
-                ptx::mbar_init(ptx::smem_u32(&ctl->stg_full[g][b]), 4);
+                ptx::mbar_init(ptx::smem_u32(&ctl->stg_full[g][b]), kOut == GPUSQ_OUT_I8 ? 8 : 4);
                 ptx::mbar_init(ptx::smem_u32(&ctl->stg_free[g][b]), 1);
             }
         ctl->abort_flag = 0;
@@ -802,10 +860,13 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             // stores must be complete before the kernel ends
             ptx::tma_store_wait_all<0>();
         } else if (kOut == GPUSQ_OUT_I8 && ptx::elect_one()) {
-            // INT8 output: staging tiles hold all 128 features of a chunk; rings 0..3 belong to the warps
-            // with that chunk index modulo 4 (rotating per tile); this lane serves rings `odd` and `odd + 2`
-            const int odd = warp - kStoreWarp0;
-            uint32_t filled_lo = 0, filled_hi = 0;         // staging tiles stored so far from ring odd / odd + 2
+            // INT8 output: a staging tile holds all 128 features of a chunk; this lane serves the ring of
+            // one chunk parity (the parity groups swap every tile)
+            const int ring = warp - kStoreWarp0;
+            const uint8_t *ring_smem = epi_smem + ring * kI8Bufs * kEpiBufBytes;
+            const uint32_t full0 = ptx::smem_u32(&ctl->stg_full[0][0]) + (uint32_t)(ring * kI8Bufs * 8);
+            const uint32_t free0 = ptx::smem_u32(&ctl->stg_free[0][0]) + (uint32_t)(ring * kI8Bufs * 8);
+            uint32_t filled = 0;                           // staging tiles stored so far
             uint32_t prev1 = 0, prev2 = 0;
             int local = 0;
             bool ok = true;
@@ -818,26 +879,22 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 if (n0 >= p.N) continue;
                 const int64_t left = p.M - m0;
                 const int nchunks = left >= h ? h / kChunkT : (int)((left + kChunkT - 1) / kChunkT);
-                for (int c = 0; c < nchunks; ++c) {
-                    const int ring = (c + local) & 3;
-                    if ((ring & 1) != odd) continue;
-                    const uint32_t count = (ring & 2) ? filled_hi : filled_lo;
-                    const uint32_t b = count % kEpiBufs;
+                for (int c = (ring + local) & 1; c < nchunks; c += 2) {
+                    const uint32_t b = filled % kI8Bufs;
                     bool to;
-                    if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->stg_full[ring][b]), (count / kEpiBufs) & 1u,
-                                                abort_flag, to)) {
+                    if (!ptx::mbar_wait_bounded(full0 + 8u * b, (filled / kI8Bufs) & 1u, abort_flag, to)) {
                         if (to) report_timeout(p, ctl, tile, 3, ring * 8 + (int)b);
                         ok = false;
                         break;
                     }
-                    ptx::tma_store_2d(&map_y, ptx::smem_u32(epi_smem + (ring * kEpiBufs + (int)b) * kEpiBufBytes), n0,
+                    ptx::tma_store_2d(&map_y, ptx::smem_u32(ring_smem + (int)b * kEpiBufBytes), n0,
                                       (int32_t)(m0 + c * kChunkT));
                     ptx::tma_store_commit();
                     ptx::tma_store_wait_read<2>();
                     if (prev2) ptx::mbar_arrive(prev2);
                     prev2 = prev1;
-                    prev1 = ptx::smem_u32(&ctl->stg_free[ring][b]);
-                    if (ring & 2) ++filled_hi; else ++filled_lo;
+                    prev1 = free0 + 8u * b;
+                    ++filled;
                 }
             }
             ptx::tma_store_wait_all<0>();
@@ -874,9 +931,9 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             e.tiles_n = tiles_n;
             e.num_tiles = num_tiles;
             if (p.act == GPUSQ_ACT_GELU)
-                e.template run<true>();
+                e.template run<true, kAmax>();
             else
-                e.template run<false>();
+                e.template run<false, kAmax>();
         } else if (kOut == GPUSQ_OUT_I8) {
             EpiI8<kTwin> e;
             e.p = &p;
@@ -1174,7 +1231,9 @@ static bool prepare_device(int kind)
                  allow_smem(gemm_i8_kernel<true, GPUSQ_OUT_I32>, b) &&
                  allow_smem(gemm_i8_kernel<true, GPUSQ_OUT_F16, false, true>, b) &&
                  allow_smem(gemm_i8_kernel<true, GPUSQ_OUT_I8, false, true>, b) &&
-                 allow_smem(gemm_i8_kernel<true, GPUSQ_OUT_I32, false, true>, b);
+                 allow_smem(gemm_i8_kernel<true, GPUSQ_OUT_I32, false, true>, b) &&
+                 allow_smem(gemm_i8_kernel<true, GPUSQ_OUT_F16, false, false, true>, b) &&
+                 allow_smem(gemm_i8_kernel<true, GPUSQ_OUT_F16, false, true, true>, b);
         } else if (kind == 1) {
             const int b = Cfg<false>::kSmemBytes;
             ok = allow_smem(gemm_i8_kernel<false, GPUSQ_OUT_F16>, b) && allow_smem(gemm_i8_kernel<false, GPUSQ_OUT_I8>, b) &&
@@ -1220,7 +1279,7 @@ static int launch_on(Kernel kernel, int smem_bytes, const CUtensorMap &map_a, co
 template <bool kSparse>
 static int launch_gemm(const int8_t *Xq, const void *Wsrc, const float *w_scale, const float *x_scale,
                        const float *bias, int act, int out_type, const float *out_scale, void *Y, int64_t M,
-                       int N, int K, int32_t *status_buf, void *stream)
+                       int N, int K, int32_t *status_buf, void *stream, float *y_absmax = nullptr)
 {
     using C = Cfg<kSparse>;
     if (!Xq || !Wsrc || !Y) return GPUSQ_ERR_NULL;
@@ -1244,6 +1303,7 @@ static int launch_gemm(const int8_t *Xq, const void *Wsrc, const float *w_scale,
     p.bias = bias;
     p.out_scale = out_scale;
     p.Y = Y;
+    p.y_absmax = y_absmax;
     p.status = status_buf;
     p.M = M;
     p.N = N;
@@ -1283,6 +1343,9 @@ static int launch_gemm(const int8_t *Xq, const void *Wsrc, const float *w_scale,
 
     // launches without a twin column run the instantiation that has no trace of it
     const int smem = C::kSmemBytes;
+    if (out_type == GPUSQ_OUT_F16 && y_absmax && kSparse)
+        return twin_col ? launch_on(gemm_i8_kernel<true, GPUSQ_OUT_F16, false, true, true>, smem, map_a, map_b, map_b2, map_e, map_y, p, clusters, stream)
+                        : launch_on(gemm_i8_kernel<true, GPUSQ_OUT_F16, false, false, true>, smem, map_a, map_b, map_b2, map_e, map_y, p, clusters, stream);
     if (out_type == GPUSQ_OUT_F16)
         return twin_col ? launch_on(gemm_i8_kernel<kSparse, GPUSQ_OUT_F16, false, true>, smem, map_a, map_b, map_b2, map_e, map_y, p, clusters, stream)
                         : launch_on(gemm_i8_kernel<kSparse, GPUSQ_OUT_F16>, smem, map_a, map_b, map_b2, map_e, map_y, p, clusters, stream);
@@ -1316,6 +1379,7 @@ static int launch_gemm_f16(const void *X, const void *Wpacked, const float *bias
     p.bias = bias;
     p.out_scale = nullptr;
     p.Y = Y;
+    p.y_absmax = nullptr;
     p.status = status_buf;
     p.M = M;
     p.N = N;
@@ -1371,6 +1435,17 @@ int gpusq_spgemm_i8(const int8_t *Xq, const void *Wpacked, const float *w_scale,
     if (Wpacked && !aligned(Wpacked, 256)) return GPUSQ_ERR_ALIGN;
     return launch_gemm<true>(Xq, Wpacked, w_scale, x_scale, bias, act, out_type, out_scale, Y, M, N, K, status_buf,
                              stream);
+}
+
+int gpusq_spgemm_i8_absmax(const int8_t *Xq, const void *Wpacked, const float *w_scale, const float *x_scale,
+                           const float *bias, int act, void *Y, float *y_absmax, int64_t M, int N, int K,
+                           int32_t *status_buf, void *stream)
+{
+    if (!y_absmax) return GPUSQ_ERR_NULL;
+    if (Wpacked && !aligned(Wpacked, 256)) return GPUSQ_ERR_ALIGN;
+    if (!aligned(y_absmax, 4)) return GPUSQ_ERR_ALIGN;
+    return launch_gemm<true>(Xq, Wpacked, w_scale, x_scale, bias, act, GPUSQ_OUT_F16, nullptr, Y, M, N, K,
+                             status_buf, stream, y_absmax);
 }
 
 int gpusq_gemm_i8_dense(const int8_t *Xq, const int8_t *Wq, const float *w_scale, const float *x_scale,

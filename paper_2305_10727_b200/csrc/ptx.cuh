@@ -189,6 +189,17 @@ __device__ __forceinline__ void stmatrix_x4_trans(uint32_t addr, uint32_t r0, ui
                  "r"(r1), "r"(r2), "r"(r3)
                  : "memory");
 }
+// four 16x8 matrices of bytes, stored transposed: matrix j takes one register per thread, whose bytes
+// are elements (row t/4, columns 2(t%4), 2(t%4)+1) and (row t/4 + 8, the same columns) -- the
+// arrangement of an accumulator fragment -- and lands as eight memory rows of 16 bytes (memory row =
+// column of the matrix, byte = row of the matrix); the address of memory row i of matrix j comes from
+// thread 8j + i.
+__device__ __forceinline__ void stmatrix_x4_trans_b8(uint32_t addr, uint32_t r0, uint32_t r1, uint32_t r2, uint32_t r3)
+{
+    asm volatile("stmatrix.sync.aligned.m16n8.x4.trans.shared.b8 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(r0),
+                 "r"(r1), "r"(r2), "r"(r3)
+                 : "memory");
+}
 // ---- CTA pairs (clusters of two) ----
 __device__ __forceinline__ uint32_t cluster_ctarank()
 {

@@ -113,8 +113,10 @@ def test_quant_act_zero_tensor_and_reused_workspace(B):
         Xq, s = B.quant_act(cu(X), workspace=ws)
         assert s.cpu().numpy()[0] == s_o
         assert np.array_equal(Xq.cpu().numpy(), Xq_o)
-    # the words of the grid-wide barrier (behind the 2048 partial maxima) are zero again after every call
-    assert not ws.cpu().numpy()[2048 * 4:2048 * 4 + 12].any()
+    # the control words and the slots of the grid-wide barrier (everything behind the 2048 words other
+    # entry points use for partial maxima) are zero again after every call
+    assert not ws.cpu().numpy()[2048 * 4:].any()
+    assert B.quant_act_status(ws) == 0
 
 
 @pytest.mark.parametrize("given", [1e-3, 0.5, 3.0, 1e-30, 1e30])
@@ -126,6 +128,34 @@ def test_quant_act_given_scale_extremes(B, given):
     Xq_o, _ = oracle.quant_act(X, x_scale=g)
     Xq, _ = B.quant_act(cu(X), x_scale=cu(np.array([g], np.float32)), scale_mode=B.SCALE_GIVEN)
     assert np.array_equal(Xq.cpu().numpy(), Xq_o)
+
+
+def test_quant_act_wait_that_runs_out_is_reported(B):
+    # A planted failure in an allowed form: the last CTA never publishes its maximum, so the bounded
+    # wait of every CTA runs out (5 ms here) and the kernel returns.  Expected: status word
+    # GPUSQ_ERR_TIMEOUT, a NaN scale (the real one is written only after every CTA came through),
+    # and, after the workspace has been zero-filled again, a correct result from the same buffers.
+    X = inputs.random_layer(77, 1576, 8, 768)["X"]
+    Xq_o, xs_o = oracle.quant_act(X)
+    Xd = cu(X)
+    ws = torch.zeros((B.quant_act_workspace(*X.shape),), dtype=torch.uint8, device="cuda")
+    Xq = torch.zeros(X.shape, dtype=torch.int8, device="cuda")
+    xs = torch.zeros((1,), dtype=torch.float32, device="cuda")
+    B.set_quant_act_wait(5_000_000, withhold_last_cta=True)
+    try:
+        B.quant_act(Xd, Xq=Xq, x_scale=xs, workspace=ws)
+        torch.cuda.synchronize()
+    finally:
+        B.set_quant_act_wait(2_000_000_000, withhold_last_cta=False)
+    assert B.quant_act_status(ws) == 7 and "TIMEOUT" in B.status_string(7)
+    assert torch.isnan(xs).all()
+    ws.zero_()
+    B.quant_act(Xd, Xq=Xq, x_scale=xs, workspace=ws)
+    assert B.quant_act_status(ws) == 0
+    assert xs.cpu().numpy()[0] == xs_o and np.array_equal(Xq.cpu().numpy(), Xq_o)
+    # and the workspace serves further calls without being touched by the caller
+    B.quant_act(Xd, Xq=Xq, x_scale=xs, workspace=ws)
+    assert B.quant_act_status(ws) == 0 and np.array_equal(Xq.cpu().numpy(), Xq_o)
 
 
 # ------------------------------------------------------------------------- GEMM
