@@ -308,6 +308,20 @@ def test_epilogue_int8_requantised(B, act, M, N, K, block_t, shrink):
         assert diff.max() <= 1 and (diff != 0).mean() < 1e-3
 
 
+@pytest.mark.parametrize("out_scale", [1e-30, 1e-17, 1e-3, 3e6, 1e9, 1e30])
+def test_epilogue_int8_extreme_output_scales(B, out_scale):
+    # supplied output scales far from the data: everything saturates, or everything rounds to zero, or the
+    # squares the kernel's range test works with leave the binary32 range; no GELU, so exact
+    M, N, K = 300, 256, 128
+    d, prep, Xq, xs = _prep(17, M, N, K)
+    acc_o = oracle.spgemm_acc(Xq, prep["vals"], prep["meta"])
+    Q_o = oracle.epilogue(acc_o, prep["w_scale"], xs, d["bias"], act=0, out_type=1, out_scale=np.float32(out_scale))
+    Q = B.spgemm_i8(cu(Xq), B.pack24(cu(prep["vals"]), cu(prep["meta"])), N, w_scale=cu(prep["w_scale"]),
+                    x_scale=cu(np.array([xs], np.float32)), bias=cu(d["bias"]), act=0, out_type=B.OUT_I8,
+                    out_scale=cu(np.array([out_scale], np.float32))).cpu().numpy()
+    assert np.array_equal(Q, Q_o)
+
+
 def test_int8_chained_mlp(B):
     # fc1 (GELU) writes requantised INT8 codes that fc2 reads with the same scale: the deployed model's
     # quantise / de-quantise chain (Sec. 2.2).  fc1's codes may differ from the oracle's by one code at
