@@ -31,4 +31,12 @@ from .oracle import (  # noqa: F401
     spgemm_f16_rows,
     epilogue_f16,
     prepare_weight_f16,
+    prune48,
+    quant_weight4,
+    compress48,
+    decompress48,
+    quant_act4,
+    spgemm48_acc,
+    prepare_weight4,
+    layer_forward4,
 )

@@ -353,6 +353,122 @@ void o_epilogue_f16(const double *acc, const float *bias, int act, uint16_t *Y, 
     }
 }
 
+/* ---- INT4 4:8 pair-wise model ---- */
+static int8_t quant_code_q(float x, float scale, float qmax)
+{
+    float q = nearbyintf(x / scale); /* ties to even */
+    if (q > qmax) q = qmax;
+    if (q < -qmax) q = -qmax;
+    return (int8_t)q;
+}
+
+void o_prune48(const float *W, float *Wp, uint8_t *mask, int N, int K)
+{
+    for (int n = 0; n < N; ++n) {
+        for (int c = 0; c < K / 8; ++c) {
+            const float *w = W + (int64_t)n * K + 8 * c;
+            double mag[4];
+            for (int p = 0; p < 4; ++p) mag[p] = fabs((double)w[2 * p]) + fabs((double)w[2 * p + 1]);
+            int p0, p1;
+            keep_two(mag, &p0, &p1);
+            for (int p = 0; p < 4; ++p) {
+                int keep = (p == p0 || p == p1);
+                Wp[(int64_t)n * K + 8 * c + 2 * p] = keep ? w[2 * p] : 0.0f;
+                Wp[(int64_t)n * K + 8 * c + 2 * p + 1] = keep ? w[2 * p + 1] : 0.0f;
+            }
+            if (mask) mask[(int64_t)n * (K / 8) + c] = (uint8_t)((1u << p0) | (1u << p1));
+        }
+    }
+}
+
+void o_quant_weight4(const float *Wp, int8_t *Wq, float *w_scale, int N, int K)
+{
+    for (int n = 0; n < N; ++n) {
+        const float *row = Wp + (int64_t)n * K;
+        float amax = 0.0f;
+        for (int k = 0; k < K; ++k) {
+            float a = fabsf(row[k]);
+            if (a > amax) amax = a;
+        }
+        float s = (amax == 0.0f) ? 1.0f : amax / 7.0f;
+        w_scale[n] = s;
+        for (int k = 0; k < K; ++k) Wq[(int64_t)n * K + k] = quant_code_q(row[k], s, 7.0f);
+    }
+}
+
+void o_compress48(const int8_t *Wq, uint8_t *vals, uint8_t *meta, int N, int K)
+{
+    memset(meta, 0, (size_t)N * (size_t)(K / 16));
+    for (int n = 0; n < N; ++n) {
+        for (int c = 0; c < K / 8; ++c) {
+            const int8_t *w = Wq + (int64_t)n * K + 8 * c;
+            double mag[4];
+            for (int p = 0; p < 4; ++p) mag[p] = fabs((double)w[2 * p]) + fabs((double)w[2 * p + 1]);
+            int p0, p1;
+            keep_two(mag, &p0, &p1);
+            const int8_t kept[4] = {w[2 * p0], w[2 * p0 + 1], w[2 * p1], w[2 * p1 + 1]};
+            uint8_t *v = vals + (int64_t)n * (K / 4) + 2 * c;
+            v[0] = (uint8_t)((kept[0] & 0xF) | ((kept[1] & 0xF) << 4));
+            v[1] = (uint8_t)((kept[2] & 0xF) | ((kept[3] & 0xF) << 4));
+            uint8_t nib = (uint8_t)(p0 | (p1 << 2));
+            meta[(int64_t)n * (K / 16) + c / 2] |= (uint8_t)(nib << (4 * (c & 1)));
+        }
+    }
+}
+
+static int8_t nibble_to_code(uint8_t nib)
+{
+    return (int8_t)((nib & 0x8) ? (int)nib - 16 : (int)nib); /* 4-bit two's complement */
+}
+
+void o_decompress48(const uint8_t *vals, const uint8_t *meta, int8_t *Wq, int N, int K)
+{
+    memset(Wq, 0, (size_t)N * (size_t)K);
+    for (int n = 0; n < N; ++n) {
+        for (int c = 0; c < K / 8; ++c) {
+            uint8_t byte = meta[(int64_t)n * (K / 16) + c / 2];
+            uint8_t nib = (uint8_t)((byte >> (4 * (c & 1))) & 0xF);
+            int p0 = nib & 3, p1 = (nib >> 2) & 3;
+            const uint8_t *v = vals + (int64_t)n * (K / 4) + 2 * c;
+            int8_t *w = Wq + (int64_t)n * K + 8 * c;
+            w[2 * p0] = nibble_to_code(v[0] & 0xF);
+            w[2 * p0 + 1] = nibble_to_code(v[0] >> 4);
+            w[2 * p1] = nibble_to_code(v[1] & 0xF);
+            w[2 * p1 + 1] = nibble_to_code(v[1] >> 4);
+        }
+    }
+}
+
+void o_quant_act4(const uint16_t *X, int8_t *Xq, float *x_scale, int scale_mode, int64_t M, int K)
+{
+    int64_t count = M * (int64_t)K;
+    float s;
+    if (scale_mode == 0) {
+        float amax = 0.0f;
+        for (int64_t i = 0; i < count; ++i) {
+            float a = fabsf(o_f16_to_f32(X[i]));
+            if (a > amax) amax = a;
+        }
+        s = (amax == 0.0f) ? 1.0f : amax / 7.0f;
+        *x_scale = s;
+    } else {
+        s = *x_scale;
+    }
+    for (int64_t i = 0; i < count; ++i) Xq[i] = quant_code_q(o_f16_to_f32(X[i]), s, 7.0f);
+}
+
+int64_t o_spgemm48_acc(const int8_t *Xq, const uint8_t *vals, const uint8_t *meta, int32_t *acc,
+                       int64_t M, int N, int K)
+{
+    int8_t *Wd = (int8_t *)malloc((size_t)N * (size_t)K);
+    if (!Wd) return -1;
+    o_decompress48(vals, meta, Wd, N, K);
+    int64_t overflow = 0;
+    for (int64_t m = 0; m < M; ++m) overflow += dot_rows(Xq + m * K, Wd, acc + m * N, N, K);
+    free(Wd);
+    return overflow;
+}
+
 double o_sqnr_db(const float *ref, const float *test, int64_t count)
 {
     double sig = 0.0, noise = 0.0;

@@ -133,6 +133,29 @@ void o_spgemm_f16_rows(const uint16_t *X, const uint16_t *vals, const uint8_t *m
  * o_epilogue; Y = binary16(y), RNE. */
 void o_epilogue_f16(const double *acc, const float *bias, int act, uint16_t *Y, int64_t count, int N);
 
+/* ---- INT4 model: Sec. 3.1 (the 4-bit format is pair-wise structured sparse at a granularity of
+ * 4:8: every chunk of eight adjacent elements of a row keeps two of its four two-wide sub-chunks,
+ * all of the other two is zero; the four kept values are stored, plus two 2-bit indices of the kept
+ * sub-chunks; 37.5 % smaller than dense INT4) and Sec. 3.4 / Table 1 (the INT4 model).
+ * Readings (paper silent): a sub-chunk's weight in the choice is |a| + |b|; the two heaviest are
+ * kept, the lower index on ties, exactly two even if zero (the keep-two rule on sub-chunks); the
+ * quantiser is the INT8 one with 7 in place of 127 (symmetric, per output channel, scale =
+ * max|row| / 7, round half to even, clamp +-7; activations per tensor alike); kept sub-chunks
+ * are re-derived from the codes when compressing.
+ * Layout: vals [N, K/4] bytes, two codes per byte in element order, the first in the low nibble
+ * (two's complement); meta [N, K/16] bytes, one nibble p0 | p1 << 2 (p0 < p1, sub-chunk indices 0..3)
+ * per chunk, the chunk with the even index in the low nibble.  K % 16 == 0.
+ * mask (nullable) [N, K/8]: bit p of the low nibble set when sub-chunk p is kept. ---- */
+void o_prune48(const float *W, float *Wp, uint8_t *mask, int N, int K);
+void o_quant_weight4(const float *Wp, int8_t *Wq, float *w_scale, int N, int K);
+void o_compress48(const int8_t *Wq, uint8_t *vals, uint8_t *meta, int N, int K);
+void o_decompress48(const uint8_t *vals, const uint8_t *meta, int8_t *Wq, int N, int K);
+/* Activations of the INT4 model: as o_quant_act with +-7 (scale = max|X| / 7). */
+void o_quant_act4(const uint16_t *X, int8_t *Xq, float *x_scale, int scale_mode, int64_t M, int K);
+/* The sparse GEMM of the 4-bit model as its definition: decompress, then 64-bit integer sums. */
+int64_t o_spgemm48_acc(const int8_t *Xq, const uint8_t *vals, const uint8_t *meta, int32_t *acc,
+                       int64_t M, int N, int K);
+
 /* binary16 <-> binary32 conversions used above (RNE narrowing). */
 uint16_t o_f32_to_f16(float f);
 float o_f16_to_f32(uint16_t h);

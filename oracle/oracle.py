@@ -71,6 +71,15 @@ def _load():
             lib.o_f32_to_f16.restype = ctypes.c_uint16
             lib.o_f16_to_f32.argtypes = [ctypes.c_uint16]
             lib.o_f16_to_f32.restype = f32
+            lib.o_prune48.argtypes = [vp, vp, vp, i32, i32]
+            lib.o_quant_weight4.argtypes = [vp, vp, vp, i32, i32]
+            lib.o_compress48.argtypes = [vp, vp, vp, i32, i32]
+            lib.o_decompress48.argtypes = [vp, vp, vp, i32, i32]
+            lib.o_quant_act4.argtypes = [vp, vp, vp, i32, i64, i32]
+            lib.o_spgemm48_acc.argtypes = [vp, vp, vp, vp, i64, i32, i32]
+            lib.o_spgemm48_acc.restype = i64
+            for name in ("o_prune48", "o_quant_weight4", "o_compress48", "o_decompress48", "o_quant_act4"):
+                getattr(lib, name).restype = None
             lib.o_sqnr_db.argtypes = [vp, vp, i64]
             lib.o_sqnr_db.restype = ctypes.c_double
             for name in ("o_prune24", "o_quant_weight", "o_compress24", "o_decompress24",
@@ -369,3 +378,89 @@ def patch_embed_forward(img, prep, P, bias=None, out_type=0, out_scale=1.0, x_sc
         acc = spgemm_acc_rows(Xq, prep["vals"], prep["meta"], rows)
     Y = epilogue(acc, prep["w_scale"], xs, bias, 0, out_type, out_scale)
     return {"imgq": imgq, "Xq": Xq, "x_scale": xs, "acc": acc, "Y": Y}
+
+
+# ---- INT4 model: pair-wise 4:8 sparsity (Sec. 3.1) ----
+
+def prune48(W, return_mask=False):
+    W = _c(W, np.float32)
+    N, K = W.shape
+    assert K % 8 == 0
+    Wp = np.empty_like(W)
+    mask = np.empty((N, K // 8), np.uint8)
+    _load().o_prune48(_p(W), _p(Wp), _p(mask), N, K)
+    return (Wp, mask) if return_mask else Wp
+
+
+def quant_weight4(Wp):
+    Wp = _c(Wp, np.float32)
+    N, K = Wp.shape
+    Wq = np.empty((N, K), np.int8)
+    s = np.empty((N,), np.float32)
+    _load().o_quant_weight4(_p(Wp), _p(Wq), _p(s), N, K)
+    return Wq, s
+
+
+def compress48(Wq):
+    Wq = _c(Wq, np.int8)
+    N, K = Wq.shape
+    assert K % 16 == 0
+    vals = np.empty((N, K // 4), np.uint8)
+    meta = np.empty((N, K // 16), np.uint8)
+    _load().o_compress48(_p(Wq), _p(vals), _p(meta), N, K)
+    return vals, meta
+
+
+def decompress48(vals, meta):
+    vals, meta = _c(vals, np.uint8), _c(meta, np.uint8)
+    N, K = vals.shape[0], vals.shape[1] * 4
+    assert meta.shape == (N, K // 16)
+    Wq = np.empty((N, K), np.int8)
+    _load().o_decompress48(_p(vals), _p(meta), _p(Wq), N, K)
+    return Wq
+
+
+def quant_act4(X, x_scale=None):
+    X = _c(X, np.float16)
+    M, K = X.shape
+    Xq = np.empty((M, K), np.int8)
+    s = np.zeros((1,), np.float32)
+    mode = 0
+    if x_scale is not None:
+        s[0] = x_scale
+        mode = 1
+    _load().o_quant_act4(_p(X.view(np.uint16)), _p(Xq), _p(s), mode, M, K)
+    return Xq, np.float32(s[0])
+
+
+def spgemm48_acc(Xq, vals, meta, threads=None):
+    Xq, vals, meta = _c(Xq, np.int8), _c(vals, np.uint8), _c(meta, np.uint8)
+    M, K = Xq.shape
+    N = vals.shape[0]
+    assert vals.shape == (N, K // 4) and meta.shape == (N, K // 16)
+    acc = np.empty((M, N), np.int32)
+    lib = _load()
+    overflow = []
+
+    def block(lo, hi):
+        overflow.append(lib.o_spgemm48_acc(_p(Xq[lo:hi]), _p(vals), _p(meta), _p(acc[lo:hi]), hi - lo, N, K))
+
+    _over_row_blocks(M, threads, block)
+    assert sum(overflow) == 0
+    return acc
+
+
+def prepare_weight4(W):
+    """Offline steps of the INT4 model: pair-wise 4:8 prune -> 4-bit quantise -> compress."""
+    Wp, mask = prune48(W, return_mask=True)
+    Wq, w_scale = quant_weight4(Wp)
+    vals, meta = compress48(Wq)
+    return {"Wp": Wp, "mask": mask, "Wq": Wq, "w_scale": w_scale, "vals": vals, "meta": meta}
+
+
+def layer_forward4(X, prep, bias=None, act=0, threads=None):
+    """Per-inference call of the INT4 model: 4-bit activation codes -> sparse GEMM -> the usual epilogue (FP16 out)."""
+    Xq, xs = quant_act4(X)
+    acc = spgemm48_acc(Xq, prep["vals"], prep["meta"], threads=threads)
+    Y = epilogue(acc, prep["w_scale"], xs, bias, act, 0, 1.0, threads=threads)
+    return {"Xq": Xq, "x_scale": xs, "acc": acc, "Y": Y}
