@@ -295,6 +295,47 @@ int gpusq_spgemm_f16(const void *X, const void *Wpacked, const float *bias, int 
                      void *Y, int64_t M, int N, int K, int32_t *status_buf, void *stream);
 
 /* ---------------------------------------------------------------------------
+ * The INT4 model.  Paper: Sec. 3.1 (for 4-bit operands the sparse format is
+ * pair-wise structured at a granularity of 4:8: of the four two-wide sub-chunks
+ * of every eight adjacent weights of a row two are kept, two are all zero; the
+ * four kept values are stored with two 2-bit sub-chunk indices; 37.5 % smaller
+ * than dense INT4) and Sec. 3.4 / Table 1 (the INT4 models, 12.7x smaller than
+ * FP32).  sm_100 tensor cores have no 4-bit integer kind, so the storage is the
+ * paper's and the arithmetic is the INT8 2:4 path's, exactly: regrouping the
+ * columns of every chunk of eight as (first elements of the four sub-chunks,
+ * then the second ones; column e -> (e % 2) * 4 + e / 2) turns the pair-wise
+ * 4:8 pattern into 2:4, and a GEMM is unchanged when weight and activation
+ * columns are permuted alike.
+ *
+ * gpusq_prune48: W [N, K] f32 -> Wp (may alias W); a sub-chunk weighs
+ *   |a| + |b| (compared as exact sums), the two heaviest of each chunk stay,
+ *   lower index on ties; mask [N, K/8] u8 nullable, bit p = sub-chunk p kept.
+ *   K % 8 == 0, W / Wp 16-byte aligned.
+ * gpusq_quant_weight4: as gpusq_quant_weight with 7 in place of 127
+ *   (w_scale[n] = max|row| / 7; codes in [-7, 7] in INT8 containers).
+ * gpusq_compress48: Wq [N, K] i8 (codes in [-7, 7]) -> vals4 [N, K/4] u8, two
+ *   codes per byte in element order, the first in the low nibble (two's
+ *   complement), and meta4 [N, K/16] u8, per chunk the nibble p0 | p1 << 2
+ *   (p0 < p1 the kept sub-chunks, re-derived from the codes), even chunk in the
+ *   low nibble.  0.3125 bytes per weight.  K % 16 == 0, Wq 16-byte aligned.
+ * gpusq_expand48: (vals4, meta4) -> vals [N, K/2] i8 and meta [N, K/8] u8 of
+ *   the SAME matrix with regrouped columns, in gpusq_compress24's format: feed
+ *   them to gpusq_pack24.  vals 8-byte aligned.
+ * gpusq_quant_act4: as gpusq_quant_act with 7 in place of 127, and the codes of
+ *   every eight columns written in the regrouped order, so that
+ *   gpusq_spgemm_i8 on (Xq, packed expanded weight) returns the 4-bit model's
+ *   sums.  Two launches with the scale computed (the first words of the
+ *   workspace are scratch, as for gpusq_patch_quant), one with it supplied.
+ */
+int gpusq_prune48(const float *W, float *Wp, uint8_t *mask, int N, int K, void *stream);
+int gpusq_quant_weight4(const float *Wp, int8_t *Wq, float *w_scale, int N, int K, void *stream);
+int gpusq_compress48(const int8_t *Wq, uint8_t *vals4, uint8_t *meta4, int N, int K, void *stream);
+int gpusq_expand48(const uint8_t *vals4, const uint8_t *meta4, int8_t *vals, uint8_t *meta, int N,
+                   int K, void *stream);
+int gpusq_quant_act4(const void *X, int8_t *Xq, float *x_scale, int scale_mode, int64_t M, int K,
+                     void *workspace, size_t ws_bytes, void *stream);
+
+/* ---------------------------------------------------------------------------
  * gpusq_gemm_i8_dense -- the same kernel and epilogue on the uncompressed
  * INT8 weight (dense tensor-core instruction): the yardstick for the paper's
  * "2x math throughput" of the sparse GEMM (Sec. 1, Sec. 3.1).

@@ -26,6 +26,7 @@ EXPORTS = (
     "gpusq_decompress24", "gpusq_packed_bytes", "gpusq_pack24", "gpusq_quant_act_workspace",
     "gpusq_quant_act", "gpusq_quant_act_static", "gpusq_patch_quant", "gpusq_spgemm_i8", "gpusq_gemm_i8_dense", "gpusq_set_block_tokens", "gpusq_set_tile_mix", "gpusq_set_quant_act_wait",
     "gpusq_spgemm_i8_absmax", "gpusq_quant_act_absmax",
+    "gpusq_prune48", "gpusq_quant_weight4", "gpusq_compress48", "gpusq_expand48", "gpusq_quant_act4",
     "gpusq_compress24_f16", "gpusq_packed_bytes_f16", "gpusq_pack24_f16", "gpusq_spgemm_f16",
 )
 
@@ -68,6 +69,11 @@ def load() -> ctypes.CDLL:
     lib.gpusq_gemm_i8_dense.argtypes = gemm_args
     lib.gpusq_spgemm_i8_absmax.argtypes = [vp, vp, vp, vp, vp, i32, vp, vp, i64, i32, i32, vp, vp]
     lib.gpusq_quant_act_absmax.argtypes = [vp, vp, vp, vp, i64, i32, vp]
+    lib.gpusq_prune48.argtypes = [vp, vp, vp, i32, i32, vp]
+    lib.gpusq_quant_weight4.argtypes = [vp, vp, vp, i32, i32, vp]
+    lib.gpusq_compress48.argtypes = [vp, vp, vp, i32, i32, vp]
+    lib.gpusq_expand48.argtypes = [vp, vp, vp, vp, i32, i32, vp]
+    lib.gpusq_quant_act4.argtypes = [vp, vp, vp, i32, i64, i32, vp, sz, vp]
     lib.gpusq_set_block_tokens.argtypes = [i32]
     lib.gpusq_set_tile_mix.argtypes = [i32, i32]
     lib.gpusq_set_quant_act_wait.argtypes = [ctypes.c_ulonglong, i32]
@@ -353,3 +359,62 @@ def spgemm_f16(X: torch.Tensor, Wpacked: torch.Tensor, N: int, bias=None, act: i
     _check(load().gpusq_spgemm_f16(_ptr(X), _ptr(Wpacked), _ptr(bias), act, out_type, _ptr(Y), M, N, K,
                                    _ptr(status_buf), _stream()), "gpusq_spgemm_f16")
     return Y
+
+
+# ---- INT4 model (pair-wise 4:8 sparsity) ----
+
+def prune48(W: torch.Tensor, want_mask: bool = False):
+    _dev(W, torch.float32, "W")
+    N, K = W.shape
+    Wp = torch.empty_like(W)
+    mask = torch.empty((N, K // 8), dtype=torch.uint8, device=W.device) if want_mask else None
+    _check(load().gpusq_prune48(_ptr(W), _ptr(Wp), _ptr(mask), N, K, _stream()), "gpusq_prune48")
+    return (Wp, mask) if want_mask else Wp
+
+
+def quant_weight4(Wp: torch.Tensor):
+    _dev(Wp, torch.float32, "Wp")
+    N, K = Wp.shape
+    Wq = torch.empty((N, K), dtype=torch.int8, device=Wp.device)
+    w_scale = torch.empty((N,), dtype=torch.float32, device=Wp.device)
+    _check(load().gpusq_quant_weight4(_ptr(Wp), _ptr(Wq), _ptr(w_scale), N, K, _stream()), "gpusq_quant_weight4")
+    return Wq, w_scale
+
+
+def compress48(Wq: torch.Tensor):
+    _dev(Wq, torch.int8, "Wq")
+    N, K = Wq.shape
+    vals4 = torch.empty((N, K // 4), dtype=torch.uint8, device=Wq.device)
+    meta4 = torch.empty((N, K // 16), dtype=torch.uint8, device=Wq.device)
+    _check(load().gpusq_compress48(_ptr(Wq), _ptr(vals4), _ptr(meta4), N, K, _stream()), "gpusq_compress48")
+    return vals4, meta4
+
+
+def expand48(vals4: torch.Tensor, meta4: torch.Tensor):
+    """(vals4, meta4) of the 4-bit format -> (vals, meta) of the 2:4 INT8 format, columns regrouped."""
+    _dev(vals4, torch.uint8, "vals4")
+    _dev(meta4, torch.uint8, "meta4")
+    N, K = vals4.shape[0], vals4.shape[1] * 4
+    vals = torch.empty((N, K // 2), dtype=torch.int8, device=vals4.device)
+    meta = torch.empty((N, K // 8), dtype=torch.uint8, device=vals4.device)
+    _check(load().gpusq_expand48(_ptr(vals4), _ptr(meta4), _ptr(vals), _ptr(meta), N, K, _stream()), "gpusq_expand48")
+    return vals, meta
+
+
+def quant_act4(X: torch.Tensor, Xq: Optional[torch.Tensor] = None, x_scale: Optional[torch.Tensor] = None,
+               scale_mode: int = SCALE_COMPUTE, workspace: Optional[torch.Tensor] = None):
+    """gpusq_quant_act4: 4-bit activation codes (INT8 containers) in the regrouped column order."""
+    _dev(X, torch.float16, "X")
+    M, K = X.shape
+    if Xq is None:
+        Xq = torch.empty((M, K), dtype=torch.int8, device=X.device)
+    if x_scale is None:
+        if scale_mode == SCALE_GIVEN:
+            raise ValueError("scale_mode GIVEN needs x_scale")
+        x_scale = torch.empty((1,), dtype=torch.float32, device=X.device)
+    if workspace is None and scale_mode == SCALE_COMPUTE:
+        workspace = torch.zeros((quant_act_workspace(M, K),), dtype=torch.uint8, device=X.device)
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(load().gpusq_quant_act4(_ptr(X), _ptr(Xq), _ptr(x_scale), scale_mode, M, K, _ptr(workspace), ws_bytes,
+                                   _stream()), "gpusq_quant_act4")
+    return Xq, x_scale

@@ -7,8 +7,8 @@
 
 namespace gpusq {
 
-// clamp(round-half-even(x / s), -127, 127) as an INT8 code, without the division and without the
-// conversion unit.
+// clamp(round-half-even(x / s), -qmax, qmax) as an INT8 code (qmax = 127; 7 for the 4-bit model),
+// without the division and without the conversion unit.
 //   Rounding: adding 1.5 * 2^23 in binary32 rounds to an integer with ties to even and leaves that
 //   integer, as a two's-complement byte, in the low byte of the sum's bit pattern; as the addend of
 //   a fused multiply-add it rounds the exact product x * c once.
@@ -25,28 +25,30 @@ constexpr float kRoundMagic = 12582912.0f;     // 1.5 * 2^23
 struct QuantScale {
     float s;            // the scale
     float2 c_lo, c_hi;  // the bracketing reciprocals, duplicated for packed math
-    float x_max;        // 127 s (kClamp)
+    float x_max;        // qmax s (kClamp)
+    float qmax;         // largest code: 127, or 7 for the 4-bit model
     bool always_divide; // 1/s is not finite
 };
 
-__device__ __forceinline__ QuantScale make_quant_scale(float s)
+__device__ __forceinline__ QuantScale make_quant_scale(float s, float qmax = 127.0f)
 {
     QuantScale a;
     a.s = s;
+    a.qmax = qmax;
     const float inv_s = __frcp_rn(s);
     const float lo = __fmul_rn(inv_s, 1.0f - 4.76837158203125e-7f), hi = __fmul_rn(inv_s, 1.0f + 4.76837158203125e-7f);
     a.c_lo = make_float2(lo, lo);
     a.c_hi = make_float2(hi, hi);
-    a.x_max = __fmul_rn(s, 127.0f);
+    a.x_max = __fmul_rn(s, qmax);
     a.always_divide = !(fabsf(inv_s) < 3.0e38f) || !(a.x_max < 3.0e38f);
     return a;
 }
 
 template <bool kClamp>
-__device__ __forceinline__ float quant_exact_sum(float x, float s)
+__device__ __forceinline__ float quant_exact_sum(float x, float s, float qmax)
 {
     float r = __fdiv_rn(x, s);
-    if (kClamp) r = fminf(fmaxf(r, -127.0f), 127.0f);
+    if (kClamp) r = fminf(fmaxf(r, -qmax), qmax);
     return r + kRoundMagic;
 }
 
@@ -66,7 +68,7 @@ __device__ __forceinline__ float2 quant2_sums(float2 f, const QuantScale &a, uin
 template <bool kClamp>
 __device__ __forceinline__ float2 quant2_exact(float2 f, const QuantScale &a)
 {
-    return make_float2(quant_exact_sum<kClamp>(f.x, a.s), quant_exact_sum<kClamp>(f.y, a.s));
+    return make_float2(quant_exact_sum<kClamp>(f.x, a.s, a.qmax), quant_exact_sum<kClamp>(f.y, a.s, a.qmax));
 }
 
 // four sums -> four codes in one word (lowest byte first)
