@@ -324,8 +324,7 @@ int gpusq_spgemm_f16(const void *X, const void *Wpacked, const float *bias, int 
  * gpusq_quant_act4: as gpusq_quant_act with 7 in place of 127, and the codes of
  *   every eight columns written in the regrouped order, so that
  *   gpusq_spgemm_i8 on (Xq, packed expanded weight) returns the 4-bit model's
- *   sums.  Two launches with the scale computed (the first words of the
- *   workspace are scratch, as for gpusq_patch_quant), one with it supplied.
+ *   sums.  Workspace, launches and status word exactly as gpusq_quant_act.
  */
 int gpusq_prune48(const float *W, float *Wp, uint8_t *mask, int N, int K, void *stream);
 int gpusq_quant_weight4(const float *Wp, int8_t *Wq, float *w_scale, int N, int K, void *stream);

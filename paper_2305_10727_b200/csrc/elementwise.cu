@@ -267,38 +267,44 @@ pack24_f16_kernel(const uint16_t *__restrict__ vals, const uint8_t *__restrict__
 }
 
 // --------------------------------------------------------------- quant_act
+// The 4-bit model (int4.cu) wants the codes of every eight columns in the order e0 e2 e4 e6 | e1 e3 e5 e7.
+__device__ __forceinline__ uint2 regrouped(uint2 q, int regroup)
+{
+    return regroup ? make_uint2(__byte_perm(q.x, q.y, 0x6420), __byte_perm(q.x, q.y, 0x7531)) : q;
+}
+
 // n_partials > 0: the scale is derived from the partial maxima and written to
 // *x_scale by block 0; absmax != NULL: it is derived from *absmax (the tensor's maximum magnitude,
 // left there by the kernel that produced X) and written; otherwise *x_scale is read.
 __global__ void __launch_bounds__(kThreads)
 act_quant_kernel(const uint4 *__restrict__ X, uint2 *__restrict__ Xq, float *x_scale,
                  const uint32_t *__restrict__ partial, int n_partials, int64_t vec8,
-                 const float *__restrict__ absmax = nullptr)
+                 const float *__restrict__ absmax = nullptr, float qmax = 127.0f, int regroup = 0)
 {
     __shared__ float red[kThreads / 32];
     float s;
     if (absmax) {
-        s = scale_from_amax(__ldg(absmax));
+        s = scale_from_amax(__ldg(absmax), qmax);
         if (blockIdx.x == 0 && threadIdx.x == 0) *x_scale = s;
     } else if (n_partials > 0) {
         uint32_t m = 0;
         for (int i = threadIdx.x; i < n_partials; i += blockDim.x) m = max(m, __ldg(partial + i));
         const uint32_t bits = (uint32_t)block_max((float)m, red);
         const float amax = __half2float(__ushort_as_half((unsigned short)bits));
-        s = scale_from_amax(amax);
+        s = scale_from_amax(amax, qmax);
         if (blockIdx.x == 0 && threadIdx.x == 0) *x_scale = s;
     } else {
         s = *x_scale;
     }
-    const QuantScale a = make_quant_scale(s);
+    const QuantScale a = make_quant_scale(s, qmax);
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     for (; i + stride < vec8; i += 2 * stride) {
         const uint4 v0 = __ldg(X + i), v1 = __ldg(X + i + stride);
-        Xq[i] = quant8_f16<true>(v0, a);
-        Xq[i + stride] = quant8_f16<true>(v1, a);
+        Xq[i] = regrouped(quant8_f16<true>(v0, a), regroup);
+        Xq[i + stride] = regrouped(quant8_f16<true>(v1, a), regroup);
     }
-    for (; i < vec8; i += stride) Xq[i] = quant8_f16<true>(__ldg(X + i), a);
+    for (; i < vec8; i += stride) Xq[i] = regrouped(quant8_f16<true>(__ldg(X + i), a), regroup);
 }
 
 // ---- patch embedding (Sec. 3.3): quantise an image batch and lay it out as the GEMM's rows ----
@@ -466,7 +472,7 @@ __device__ __forceinline__ bool mbar_try_wait_parity0(uint32_t bar)
 
 __global__ void __launch_bounds__(kFusedThreads, 1)
 act_quant_fused_kernel(const uint4 *__restrict__ X, uint2 *__restrict__ Xq, float *x_scale,
-                       uint32_t *ws, int64_t vec8, unsigned long long wait_ns, int withhold)
+                       uint32_t *ws, int64_t vec8, unsigned long long wait_ns, int withhold, float qmax, int regroup)
 {
     extern __shared__ __align__(128) uint4 cache[];
     __shared__ float red[kFusedThreads / 32];
@@ -583,22 +589,22 @@ act_quant_fused_kernel(const uint4 *__restrict__ X, uint2 *__restrict__ Xq, floa
         if (atomicAdd(ws + kWsDone, 1u) == gridDim.x - 1) {
             __stcg(reinterpret_cast<uint2 *>(bar_word), make_uint2(0u, 0u));
             __stcg(ws + kWsDone, 0u);
-            *x_scale = scale_from_amax(__half2float(__ushort_as_half((unsigned short)all)));
+            *x_scale = scale_from_amax(__half2float(__ushort_as_half((unsigned short)all)), qmax);
         }
     }
-    const float s = scale_from_amax(__half2float(__ushort_as_half((unsigned short)all)));
-    const QuantScale a = make_quant_scale(s);
+    const float s = scale_from_amax(__half2float(__ushort_as_half((unsigned short)all)), qmax);
+    const QuantScale a = make_quant_scale(s, qmax);
 
     // 3. quantise the slice: what was kept, from shared memory; the rest, from L2 / HBM
-    for (i = tid; i < n_kept; i += kFusedThreads) __stcs(Xqs + i, quant8_f16<false>(cache[i], a));
+    for (i = tid; i < n_kept; i += kFusedThreads) __stcs(Xqs + i, regrouped(quant8_f16<false>(cache[i], a), regroup));
     for (; i + 3 * kFusedThreads < n; i += 4 * kFusedThreads) {
         uint4 v[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) v[u] = __ldg(Xs + i + u * kFusedThreads);
 #pragma unroll
-        for (int u = 0; u < 4; ++u) __stcs(Xqs + i + u * kFusedThreads, quant8_f16<false>(v[u], a));
+        for (int u = 0; u < 4; ++u) __stcs(Xqs + i + u * kFusedThreads, regrouped(quant8_f16<false>(v[u], a), regroup));
     }
-    for (; i < n; i += kFusedThreads) __stcs(Xqs + i, quant8_f16<false>(__ldg(Xs + i), a));
+    for (; i < n; i += kFusedThreads) __stcs(Xqs + i, regrouped(quant8_f16<false>(__ldg(Xs + i), a), regroup));
 }
 
 // ---- library-owned scratch for gpusq_quant_act_static ----
@@ -743,8 +749,9 @@ size_t gpusq_quant_act_workspace(int64_t M, int K)
     return (size_t)(kMaxPartials + kWorkspaceExtra) * sizeof(uint32_t);
 }
 
-int gpusq_quant_act(const void *X, int8_t *Xq, float *x_scale, int scale_mode, int64_t M, int K,
-                    void *workspace, size_t ws_bytes, void *stream)
+// gpusq_quant_act (qmax 127) and gpusq_quant_act4 (qmax 7, codes of every eight columns regrouped)
+static int quant_act_common(const void *X, int8_t *Xq, float *x_scale, int scale_mode, int64_t M, int K,
+                            void *workspace, size_t ws_bytes, void *stream, float qmax, int regroup)
 {
     static_assert(GPUSQ_QUANT_ACT_STATUS_OFFSET == kWsStatus * sizeof(uint32_t), "status word as documented");
     if (!X || !Xq || !x_scale) return GPUSQ_ERR_NULL;
@@ -797,15 +804,28 @@ int gpusq_quant_act(const void *X, int8_t *Xq, float *x_scale, int scale_mode, i
         const int withhold = g_withhold_slot.load(std::memory_order_relaxed);
         if (cudaLaunchKernelEx(&cfg, act_quant_fused_kernel, reinterpret_cast<const uint4 *>(X),
                                reinterpret_cast<uint2 *>(Xq), x_scale, reinterpret_cast<uint32_t *>(workspace), vec8,
-                               wait_ns, withhold) != cudaSuccess) {
+                               wait_ns, withhold, qmax, regroup) != cudaSuccess) {
             (void)cudaGetLastError();
             return GPUSQ_ERR_CUDA;
         }
         return GPUSQ_OK;
     }
     act_quant_kernel<<<grid_for(ceil_div(vec8, 2), 8), kThreads, 0, s>>>(
-        reinterpret_cast<const uint4 *>(X), reinterpret_cast<uint2 *>(Xq), x_scale, nullptr, 0, vec8);
+        reinterpret_cast<const uint4 *>(X), reinterpret_cast<uint2 *>(Xq), x_scale, nullptr, 0, vec8, nullptr, qmax,
+        regroup);
     return launch_status();
+}
+
+int gpusq_quant_act(const void *X, int8_t *Xq, float *x_scale, int scale_mode, int64_t M, int K,
+                    void *workspace, size_t ws_bytes, void *stream)
+{
+    return quant_act_common(X, Xq, x_scale, scale_mode, M, K, workspace, ws_bytes, stream, 127.0f, 0);
+}
+
+int gpusq_quant_act4(const void *X, int8_t *Xq, float *x_scale, int scale_mode, int64_t M, int K,
+                     void *workspace, size_t ws_bytes, void *stream)
+{
+    return quant_act_common(X, Xq, x_scale, scale_mode, M, K, workspace, ws_bytes, stream, 7.0f, 1);
 }
 
 int gpusq_quant_act_absmax(const void *X, int8_t *Xq, float *x_scale, const float *absmax, int64_t M, int K,

@@ -7,7 +7,7 @@
 // four sub-chunks and then the second ones (column e -> (e % 2) * 4 + e / 2) turns "two of four
 // sub-chunks kept" into "two of every four columns kept".  A GEMM does not change when weight and
 // activation columns are permuted alike, so gpusq_expand48 writes the weight in that column order as
-// an ordinary 2:4 INT8 operand, gpusq_quant_act4 writes the 4-bit activation codes in the same
+// an ordinary 2:4 INT8 operand, gpusq_quant_act4 (elementwise.cu) writes the 4-bit activation codes in the same
 // order, and gpusq_pack24 + gpusq_spgemm_i8 do the rest.  The 2x math rate 4-bit tensor cores gave
 // the paper's GPUs is not available; the storage saving and the results are.
 #include "prep_common.cuh"
@@ -113,32 +113,6 @@ expand48_kernel(const uint32_t *__restrict__ vals4, const uint8_t *__restrict__ 
     }
 }
 
-// --------------------------------------------------------------- quant_act4
-// Codes in [-7, 7], written in the regrouped column order (bytes e0 e2 e4 e6 | e1 e3 e5 e7 of every
-// eight).  n_partials > 0: scale = maximum / 7 from the partial maxima; else *x_scale is read.
-__global__ void __launch_bounds__(kThreads)
-act_quant4_kernel(const uint4 *__restrict__ X, uint2 *__restrict__ Xq, float *x_scale,
-                  const uint32_t *__restrict__ partial, int n_partials, int64_t vec8)
-{
-    __shared__ float red[kThreads / 32];
-    float s;
-    if (n_partials > 0) {
-        uint32_t m = 0;
-        for (int i = threadIdx.x; i < n_partials; i += blockDim.x) m = max(m, __ldg(partial + i));
-        const uint32_t bits = (uint32_t)block_max((float)m, red);
-        s = scale_from_amax(__half2float(__ushort_as_half((unsigned short)bits)), 7.0f);
-        if (blockIdx.x == 0 && threadIdx.x == 0) *x_scale = s;
-    } else {
-        s = *x_scale;
-    }
-    const QuantScale a = make_quant_scale(s, 7.0f);
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < vec8; i += stride) {
-        const uint2 q = quant8_f16<true>(__ldg(X + i), a);
-        Xq[i] = make_uint2(__byte_perm(q.x, q.y, 0x6420), __byte_perm(q.x, q.y, 0x7531));
-    }
-}
-
 }  // namespace gpusq
 
 using namespace gpusq;
@@ -191,35 +165,6 @@ int gpusq_expand48(const uint8_t *vals4, const uint8_t *meta4, int8_t *vals, uin
     expand48_kernel<<<grid_for(pairs, 8), kThreads, 0, (cudaStream_t)stream>>>(
         reinterpret_cast<const uint32_t *>(vals4), meta4, reinterpret_cast<uint2 *>(vals),
         reinterpret_cast<uint16_t *>(meta), pairs);
-    return launch_status();
-}
-
-int gpusq_quant_act4(const void *X, int8_t *Xq, float *x_scale, int scale_mode, int64_t M, int K, void *workspace,
-                     size_t ws_bytes, void *stream)
-{
-    if (!X || !Xq || !x_scale) return GPUSQ_ERR_NULL;
-    if (M <= 0 || K <= 0 || K % 8) return GPUSQ_ERR_SHAPE;
-    if (scale_mode != GPUSQ_SCALE_COMPUTE && scale_mode != GPUSQ_SCALE_GIVEN) return GPUSQ_ERR_ARG;
-    if (!aligned(X, 16) || !aligned(Xq, 16)) return GPUSQ_ERR_ALIGN;
-    if (scale_mode == GPUSQ_SCALE_COMPUTE) {
-        if (!workspace || ws_bytes < gpusq_quant_act_workspace(M, K)) return GPUSQ_ERR_WORKSPACE;
-        if (!aligned(workspace, 16)) return GPUSQ_ERR_ALIGN;
-    }
-    if (int st = check_arch()) return st;
-    const int64_t vec8 = M * (int64_t)K / 8;
-    cudaStream_t s = (cudaStream_t)stream;
-    uint32_t *partial = reinterpret_cast<uint32_t *>(workspace);
-    int n_partials = 0;
-    if (scale_mode == GPUSQ_SCALE_COMPUTE) {
-        // the first words of the workspace, every one written before it is read; the words
-        // gpusq_quant_act keeps zero are not touched
-        n_partials = grid_for(ceil_div(vec8, 4), 8);
-        if (n_partials > kMaxPartials) n_partials = kMaxPartials;
-        act_absmax_kernel<<<n_partials, kThreads, 0, s>>>(reinterpret_cast<const uint4 *>(X), partial, vec8);
-        if (int st = launch_status()) return st;
-    }
-    act_quant4_kernel<<<grid_for(vec8, 8), kThreads, 0, s>>>(reinterpret_cast<const uint4 *>(X),
-                                                            reinterpret_cast<uint2 *>(Xq), x_scale, partial, n_partials, vec8);
     return launch_status();
 }
 
