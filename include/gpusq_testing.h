@@ -32,6 +32,15 @@ int gpusq_set_tile_mix(int block_t, int n_big);
  * faults or hangs: the waits end at the bound. */
 int gpusq_set_quant_act_wait(unsigned long long limit_ns, int withhold_last_cta);
 
+/* The same for the GEMM kernels: bound of every device-side wait in microseconds
+ * (default 2 s) and, with withhold_loads != 0, a planted failure in an allowed
+ * form: the producers of the first CTA pair stop before the last k block of
+ * their first tile, so the MMA issuer's bounded wait for that block runs out;
+ * it raises the pair's abort flag, writes {GPUSQ_ERR_TIMEOUT, tile, role,
+ * stage} to status_buf, every role of the pair leaves its loop, and the kernel
+ * returns.  The other pairs finish their tiles.  Nothing faults or hangs. */
+int gpusq_set_gemm_wait(unsigned limit_us, int withhold_loads);
+
 #ifdef __cplusplus
 }
 #endif

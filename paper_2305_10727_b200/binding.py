@@ -24,7 +24,7 @@ SCALE_COMPUTE, SCALE_GIVEN = 0, 1
 EXPORTS = (
     "gpusq_status_string", "gpusq_prune24", "gpusq_quant_weight", "gpusq_compress24",
     "gpusq_decompress24", "gpusq_packed_bytes", "gpusq_pack24", "gpusq_quant_act_workspace",
-    "gpusq_quant_act", "gpusq_quant_act_static", "gpusq_patch_quant", "gpusq_spgemm_i8", "gpusq_gemm_i8_dense", "gpusq_set_block_tokens", "gpusq_set_tile_mix", "gpusq_set_quant_act_wait",
+    "gpusq_quant_act", "gpusq_quant_act_static", "gpusq_patch_quant", "gpusq_spgemm_i8", "gpusq_gemm_i8_dense", "gpusq_set_block_tokens", "gpusq_set_tile_mix", "gpusq_set_quant_act_wait", "gpusq_set_gemm_wait",
     "gpusq_spgemm_i8_absmax", "gpusq_quant_act_absmax",
     "gpusq_prune48", "gpusq_quant_weight4", "gpusq_compress48", "gpusq_expand48", "gpusq_quant_act4",
     "gpusq_compress24_f16", "gpusq_packed_bytes_f16", "gpusq_pack24_f16", "gpusq_spgemm_f16",
@@ -77,6 +77,7 @@ def load() -> ctypes.CDLL:
     lib.gpusq_set_block_tokens.argtypes = [i32]
     lib.gpusq_set_tile_mix.argtypes = [i32, i32]
     lib.gpusq_set_quant_act_wait.argtypes = [ctypes.c_ulonglong, i32]
+    lib.gpusq_set_gemm_wait.argtypes = [ctypes.c_uint, i32]
     lib.gpusq_compress24_f16.argtypes = [vp, vp, vp, i32, i32, vp]
     lib.gpusq_packed_bytes_f16.argtypes = [i32, i32]
     lib.gpusq_packed_bytes_f16.restype = sz
@@ -205,6 +206,11 @@ def quant_act_status(workspace: torch.Tensor) -> int:
 def set_quant_act_wait(limit_ns: int, withhold_last_cta: bool = False) -> None:
     """Test hook (gpusq_testing.h): bound of the one-launch kernel's waits; optionally plant an arrival that never comes."""
     _check(load().gpusq_set_quant_act_wait(int(limit_ns), 1 if withhold_last_cta else 0), "gpusq_set_quant_act_wait")
+
+
+def set_gemm_wait(limit_us: int, withhold_loads: bool = False) -> None:
+    """Test hook (gpusq_testing.h): bound of the GEMM kernels' waits; optionally plant loads that never come."""
+    _check(load().gpusq_set_gemm_wait(int(limit_us), 1 if withhold_loads else 0), "gpusq_set_gemm_wait")
 
 
 def quant_act_static(X: torch.Tensor, Xq: Optional[torch.Tensor] = None, x_scale: Optional[torch.Tensor] = None,

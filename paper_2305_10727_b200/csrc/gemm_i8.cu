@@ -103,6 +103,7 @@ struct Ctl {
     uint64_t stg_free[kEpiGroups][kEpiBufs];     // staging tile read by its TMA store
     uint32_t tmem_base;
     uint32_t abort_flag;
+    uint32_t wait_us;       // directly behind the flag: the bounded waits read their limit from here
 };
 
 struct GemmParams {
@@ -125,6 +126,8 @@ struct GemmParams {
     int num_tiles;
     int twin_n0;    // first feature of the twin column (256 pair_cols)
     int oob_row;    // a row coordinate beyond the weight tensor: loads from there fill with zeros
+    uint32_t wait_us;   // limit of every device-side wait, microseconds
+    int withhold;       // test hook: the first cluster's producers stop before the last k block of their first tile
 };
 
 // Where a tile sits.  Normally a pair shares `h` tokens and CTA `rank` owns 128 of the pair's 256
@@ -644,6 +647,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 ptx::mbar_init(ptx::smem_u32(&ctl->stg_free[g][b]), 1);
             }
         ctl->abort_flag = 0;
+        ctl->wait_us = p.wait_us;
         ptx::fence_barrier_init();
         ptx::prefetch_tensormap(&map_a);
         ptx::prefetch_tensormap(&map_b);
@@ -688,6 +692,11 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 // bytes both CTAs together bring in per stage
                 const uint32_t stage_tx = 2u * (uint32_t)(C::kABytes + C::kBAtoms * half_t * 128 + C::kMetaBytes);
                 for (int ks = 0; ks < num_kb; ++ks) {
+                    if (p.withhold && tile == 0 && ks == num_kb - 1) {
+                        // planted failure (test hook): these loads never come, the MMA issuer's wait runs out
+                        ok = false;
+                        break;
+                    }
                     // twin tiles: pass `seg` of the k blocks runs against the token tile of CTA `seg`, whose
                     // weights sit in that CTA only (the other one loads zeros from beyond the tensor)
                     const int seg = twin ? ks / k_blocks : 0;
@@ -731,9 +740,9 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 // do not leave while bulk copies may still land in the pair's shared memory
                 for (int s = 0; s < C::kStages; ++s) {
                     if (issued & (1u << s)) {
-                        uint32_t none = 0;
+                        uint32_t none[2] = {0u, p.wait_us};
                         bool to;
-                        (void)ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->full[s]), (last_parity >> s) & 1u, &none, to);
+                        (void)ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->full[s]), (last_parity >> s) & 1u, none, to);
                     }
                 }
             }
@@ -809,9 +818,9 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             if (*abort_flag) {
                 // let every MMA issued so far retire before tensor memory is released
                 ptx::tc_commit(ptx::smem_u32(&ctl->drain));
-                uint32_t none = 0;
+                uint32_t none[2] = {0u, p.wait_us};
                 bool to;
-                (void)ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->drain), 0, &none, to);
+                (void)ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->drain), 0, none, to);
             }
         }
     } else if (warp >= kStoreWarp0) {
@@ -1054,6 +1063,8 @@ static bool make_map_y_f16(CUtensorMap *map, void *base, uint64_t M, uint64_t N)
 // testing hooks (gpusq_testing.h): a forced tile height, and a forced number of full-height token tiles
 static std::atomic<int> g_block_t_override{0};
 static std::atomic<int> g_n_big_override{-1};
+static std::atomic<unsigned> g_wait_us{ptx::kDefaultWaitUs};
+static std::atomic<int> g_withhold_loads{0};
 
 // How the token axis is cut into tiles: tok_tiles token tiles, the first n_big of them block_t tokens
 // high, the others block_t - 32.
@@ -1181,6 +1192,8 @@ static bool set_tiling(GemmParams &p, int64_t M, int N, int K_cost, int clusters
     p.num_tiles = (int)tiles;
     p.twin_n0 = p.pair_cols * kPairF;
     p.oob_row = round_up(N, kPairF);  // beyond the packed rows (N rounded up) and the plain ones (N) alike
+    p.wait_us = g_wait_us.load(std::memory_order_relaxed);
+    p.withhold = g_withhold_loads.load(std::memory_order_relaxed);
     return true;
 }
 
@@ -1461,6 +1474,14 @@ int gpusq_set_block_tokens(int block_t)
     if (block_t != 0 && (block_t < 32 || block_t > kMaxBlockT || block_t % 32)) return GPUSQ_ERR_ARG;
     g_block_t_override.store(block_t, std::memory_order_relaxed);
     g_n_big_override.store(-1, std::memory_order_relaxed);
+    return GPUSQ_OK;
+}
+
+int gpusq_set_gemm_wait(unsigned limit_us, int withhold_loads)
+{
+    if (limit_us == 0) return GPUSQ_ERR_ARG;
+    g_wait_us.store(limit_us, std::memory_order_relaxed);
+    g_withhold_loads.store(withhold_loads ? 1 : 0, std::memory_order_relaxed);
     return GPUSQ_OK;
 }
 

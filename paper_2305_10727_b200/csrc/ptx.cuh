@@ -73,8 +73,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 
-// Bounded wait: gives up after `kWaitLimitNs` of wall time, or as soon as another
-// thread of the CTA has raised *abort_flag.  Returns false on either; the
+// Bounded wait: gives up after the time limit, or as soon as another thread of the CTA has raised
+// *abort_flag.  The limit, in microseconds, is the word behind the flag (abort_flag[1]; 2 s unless the
+// test hook shortens it).  Returns false on either; the
 // caller that timed out raises the flag itself.  The common case (the phase
 // is complete already) costs one try and one branch; the retry loop is kept
 // out of line so that it does not bloat the callers' instruction streams.
@@ -82,7 +83,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 // time has passed, so a waiting warp issues a few instructions per microsecond
 // and wakes as soon as the barrier flips; the flag and the clock are looked at
 // after every `kTriesPerCheck` expired tries.
-constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s
+constexpr uint32_t kDefaultWaitUs = 2000000u;      // 2 s
 constexpr uint32_t kSuspendHintNs = 1000;
 __device__ __forceinline__ bool mbar_try_wait_32(uint32_t bar, uint32_t parity)
 {
@@ -114,7 +115,7 @@ __device__ __noinline__ int mbar_wait_slow(uint32_t bar, uint32_t parity, volati
     for (;;) {
         if (mbar_try_wait_32(bar, parity)) return 0;
         if (*abort_flag) return 1;
-        if (globaltimer_ns() - t0 > kWaitLimitNs) return 2;
+        if (globaltimer_ns() - t0 > (uint64_t)abort_flag[1] * 1000ull) return 2;
     }
 }
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,

@@ -224,6 +224,31 @@ def test_mixed_tile_heights(B, M, N, K, block_t, n_big):
     assert np.array_equal(Q, Q_o)
 
 
+def test_gemm_wait_that_runs_out_is_reported(B):
+    # A planted failure in an allowed form: the first CTA pair's loads for the last k block of its first tile
+    # are never issued, so the MMA issuer's bounded wait (5 ms here) runs out.  Expected: status_buf =
+    # {GPUSQ_ERR_TIMEOUT, tile 0, role 1 (MMA issuer), stage}, the kernel returns, and the next call on
+    # the same buffers is correct (the context is intact, tensor memory was released).
+    M, N, K = 1576, 768, 192
+    d, prep, Xq, xs = _prep(123, M, N, K)
+    acc_o = oracle.spgemm_acc(Xq, prep["vals"], prep["meta"])
+    Wpk = B.pack24(cu(prep["vals"]), cu(prep["meta"]))
+    Xd = cu(Xq)
+    status = torch.zeros(4, dtype=torch.int32, device="cuda")
+    B.set_gemm_wait(5000, withhold_loads=True)
+    try:
+        B.spgemm_i8(Xd, Wpk, N, out_type=B.OUT_I32, status_buf=status)
+        torch.cuda.synchronize()
+    finally:
+        B.set_gemm_wait(2_000_000, withhold_loads=False)
+    st = status.cpu().tolist()
+    assert st[0] == 7 and st[1] == 0 and st[2] == 1, st
+    status.zero_()
+    Y = B.spgemm_i8(Xd, Wpk, N, out_type=B.OUT_I32, status_buf=status)
+    assert status.cpu().tolist() == [0, 0, 0, 0]
+    assert np.array_equal(Y.cpu().numpy(), acc_o)
+
+
 def test_spgemm_extreme_codes_do_not_overflow(B):
     # every kept code and every activation at +-127, K = 5120: |acc| = 127^2 * K / 2
     M, N, K = 40, 128, 5120
