@@ -57,14 +57,18 @@ constexpr int kPairF = 2 * kBlockF; // features per CTA pair and tile
 constexpr int kBlockK = 128;        // K per stage
 constexpr int kMaxBlockT = 224;     // tokens per tile (runtime value, multiple of 32)
 constexpr int kChunkT = 32;         // tokens per epilogue chunk
-constexpr int kEpiWarps = 16;
-constexpr int kStoreWarp0 = 2 + kEpiWarps;   // first of the two store warps
-constexpr int kNumThreads = 32 * (kStoreWarp0 + 2);
+// Chunk phases of the epilogue: eight epilogue warps per phase.  Two (16 warps of 96 registers) is
+// what is built; one (8 warps) is as fast without GELU and slower with it or with INT8 output, three
+// (24 warps of 72 registers, two staging tiles per group) is 1.5x slower on every layer.
+#ifndef GPUSQ_PHASES
+#define GPUSQ_PHASES 2
+#endif
+constexpr int kMaxPhases = 3;       // chunk phases: eight epilogue warps (128 features) per phase
 constexpr int kTmemCols = 512;
 constexpr int kAccStride = 256;     // column offset of the second accumulator
 constexpr int kMetaCol = 224;       // metadata slots: 4 columns per stage from here (below the second accumulator)
-constexpr int kEpiGroups = 4;       // groups of four epilogue warps: 64 features x every other chunk
-constexpr int kEpiBufs = 3;         // staging tiles per group (two in the FP16 model, which needs the room for a fourth stage)
+constexpr int kMaxEpiGroups = 2 * kMaxPhases;   // groups of four epilogue warps: 64 features x chunk phase
+constexpr int kMaxEpiBufs = 3;                  // staging tiles per group, at most
 constexpr int kEpiBufBytes = kChunkT * 128;           // [32 tokens][64 features] f16
 
 // kHalf: the FP16 2:4 sparse model (binary16 operands, FP32 accumulators) instead of INT8.  A stage
@@ -79,7 +83,15 @@ struct Cfg {
     static constexpr int kMetaBytes = kSparse ? 2048 : 0;
     static constexpr int kStageBytes = kABytes + kBBytes + kMetaBytes;
     static constexpr int kStages = kHalf ? 4 : kSparse ? 7 : 5;
-    static constexpr int kEpiBufs = kHalf ? 2 : gpusq::kEpiBufs;
+    // Epilogue warps: eight per chunk phase (the warps of phase p take the chunks c of a tile with
+    // (p + tile count) mod kPhases == c mod kPhases).
+    static constexpr int kPhases = kHalf ? 2 : GPUSQ_PHASES;
+    static constexpr int kEpiWarps = 8 * kPhases;
+    static constexpr int kStoreWarp0 = 2 + kEpiWarps;          // first of the two store warps
+    static constexpr int kThreads = 32 * (kStoreWarp0 + 2);
+    static constexpr int kEpiGroups = 2 * kPhases;             // 64 features x chunk phase: four warps share a staging tile
+    static constexpr int kEpiBufs = kPhases == 3 ? 2 : kPhases == 1 ? 6 : kHalf ? 2 : 3;      // staging tiles per group
+    static constexpr int kI8Bufs = 2 * kEpiBufs;               // INT8 output: one ring per phase over the same shared memory
     static constexpr int kEpiBytes = kEpiGroups * kEpiBufs * kEpiBufBytes;
     static constexpr int kCtlBytes = 1024;
     static constexpr int kSmemBytes = kStages * kStageBytes + kEpiBytes + kCtlBytes + 1024 /* alignment slack */;
@@ -99,8 +111,8 @@ struct Ctl {
     uint64_t tmem_full[2];
     uint64_t tmem_empty[2];
     uint64_t drain;
-    uint64_t stg_full[kEpiGroups][kEpiBufs];     // staging tile written by its four warps
-    uint64_t stg_free[kEpiGroups][kEpiBufs];     // staging tile read by its TMA store
+    uint64_t stg_full[kMaxEpiGroups * kMaxEpiBufs];     // staging tile written by its four warps (flat: group * bufs + tile)
+    uint64_t stg_free[kMaxEpiGroups * kMaxEpiBufs];     // staging tile read by its TMA store
     uint32_t tmem_base;
     uint32_t abort_flag;
     uint32_t wait_us;       // directly behind the flag: the bounded waits read their limit from here
@@ -240,7 +252,7 @@ __device__ __forceinline__ float2 gelu_pair(float2 y)
 // ahead), issue the next one, convert / scale / activate 16 values per thread, wait for a free
 // staging tile, two stmatrix, proxy fence, arrive on the tile's full barrier.  The loop is written
 // for few instructions per chunk: whatever can be precomputed or advanced incrementally is.
-template <bool kAccFloat, int kBufs, bool kTwin>
+template <bool kAccFloat, int kBufs, int kPhases, bool kTwin>
 struct EpiF16 {
     const GemmParams *p;
     Ctl *ctl;
@@ -330,7 +342,7 @@ struct EpiF16 {
     {
         const int quarter = warp & 3;                      // tensor-memory lanes [32q, 32q+32) are this warp's to read
         const int half = ((warp - 2) >> 2) & 1;            // which 16 of them
-        const int par = (warp - 2) >> 3;                   // which chunks: every other one
+        const int par = (warp - 2) >> 3;                   // which chunks: every kPhases-th one
         const int nofs = quarter * 32 + 16 * half + (lane >> 2);       // this thread's first feature in the CTA's 128
         amax = 0.0f;
         {
@@ -393,9 +405,9 @@ struct EpiF16 {
                 const int64_t left = M - m0;               // > 0
                 nchunks = left >= h ? h / kChunkT : (int)((left + kChunkT - 1) / kChunkT);
             }
-            // this warp's chunks of the tile: c0, c0 + 2, ...; the two parity groups swap every tile
-            const int c0 = (par + local) & 1;
-            int mine = (nchunks - c0 + 1) >> 1;            // how many of them
+            // this warp's chunks of the tile: c0, c0 + kPhases, ...; the phases rotate every tile
+            const int c0 = (par + local) % kPhases;
+            int mine = (nchunks - c0 + kPhases - 1) / kPhases;         // how many of them
             if (mine <= 0) {
                 release(acc);
                 continue;
@@ -408,14 +420,14 @@ struct EpiF16 {
             const int64_t ahead = M - m0 - (int64_t)c0 * kChunkT;
             int rows = ahead > 4 * kMaxBlockT ? 4 * kMaxBlockT : (int)ahead;
             for (;;) {
-                taddr += 2 * kChunkT;
+                taddr += kPhases * kChunkT;
                 if (!step<kGelu, kAmax>(v0, v1, --mine ? taddr : 0u, acc, tile, rows)) return;
                 if (!mine) break;
-                rows -= 2 * kChunkT;
-                taddr += 2 * kChunkT;
+                rows -= kPhases * kChunkT;
+                taddr += kPhases * kChunkT;
                 if (!step<kGelu, kAmax>(v1, v0, --mine ? taddr : 0u, acc, tile, rows)) return;
                 if (!mine) break;
-                rows -= 2 * kChunkT;
+                rows -= kPhases * kChunkT;
             }
         }
         if (kAmax) {
@@ -436,9 +448,7 @@ struct EpiF16 {
 // (stmatrix m16n8 b8, transposed): one instruction per chunk writes the warp's 32 tokens x 16 features
 // as 16-byte row pieces into a 128-byte-swizzled [32 tokens][128 features] staging tile that the
 // eight warps of the same chunk parity fill together; a TMA store writes full 128-byte rows of Y.
-constexpr int kI8Bufs = kEpiGroups * kEpiBufs / 2;      // staging tiles per chunk parity (the same shared memory, two rings)
-
-template <bool kTwin>
+template <int kI8Bufs, int kPhases, bool kTwin>
 struct EpiI8 {
     const GemmParams *p;
     Ctl *ctl;
@@ -516,14 +526,14 @@ struct EpiI8 {
     {
         const int quarter = warp & 3;                      // tensor-memory lanes [32q, 32q+32) are this warp's to read
         const int half = ((warp - 2) >> 2) & 1;            // which 16 of them
-        const int par = (warp - 2) >> 3;                   // which chunks: every other one
+        const int par = (warp - 2) >> 3;                   // which chunks: every kPhases-th one
         const int nofs = quarter * 32 + 16 * half + (lane >> 2);
         // this lane's address in the matrix store: row = token `lane` of the chunk, the warp's 16-byte column
         stm_off = (uint32_t)(lane * 128 + (((2 * quarter + half) ^ (lane & 7)) << 4));
         // the barriers of the staging tiles, taken as one array: ring `par` uses entries par * kI8Bufs ...
         ring0 = ptx::smem_u32(epi_smem + par * kI8Bufs * kEpiBufBytes);
-        full0 = ptx::smem_u32(&ctl->stg_full[0][0]) + (uint32_t)(par * kI8Bufs * 8);
-        free0 = ptx::smem_u32(&ctl->stg_free[0][0]) + (uint32_t)(par * kI8Bufs * 8);
+        full0 = ptx::smem_u32(&ctl->stg_full[0]) + (uint32_t)(par * kI8Bufs * 8);
+        free0 = ptx::smem_u32(&ctl->stg_free[0]) + (uint32_t)(par * kI8Bufs * 8);
         buf_addr = ring0;
         full_bar = full0;
         free_bar = free0;
@@ -577,8 +587,8 @@ struct EpiI8 {
                 const int64_t left = M - m0;
                 nchunks = left >= h ? h / kChunkT : (int)((left + kChunkT - 1) / kChunkT);
             }
-            const int c0 = (par + local) & 1;
-            int mine = (nchunks - c0 + 1) >> 1;
+            const int c0 = (par + local) % kPhases;
+            int mine = (nchunks - c0 + kPhases - 1) / kPhases;
             if (mine <= 0) {
                 release(acc);
                 continue;
@@ -588,10 +598,10 @@ struct EpiI8 {
             uint32_t v0[16], v1[16];
             ptx::tmem_ld_16x256b_x4(taddr, v0);
             for (;;) {
-                taddr += 2 * kChunkT;
+                taddr += kPhases * kChunkT;
                 if (!step<kGelu>(v0, v1, --mine ? taddr : 0u, acc, tile)) return;
                 if (!mine) break;
-                taddr += 2 * kChunkT;
+                taddr += kPhases * kChunkT;
                 if (!step<kGelu>(v1, v0, --mine ? taddr : 0u, acc, tile)) return;
                 if (!mine) break;
             }
@@ -604,7 +614,7 @@ struct EpiI8 {
 // kAmax: the FP16 epilogue also merges max |Y| into a device word (its own instantiation, so that the
 // ordinary kernel's register allocation is untouched)
 template <bool kSparse, int kOut, bool kHalf = false, bool kTwin = false, bool kAmax = false>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kNumThreads, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__((Cfg<kSparse, kHalf>::kThreads), 1)
 gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_b2, const __grid_constant__ CUtensorMap map_e,
                const __grid_constant__ CUtensorMap map_y, const GemmParams p)
@@ -616,6 +626,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     uint8_t *epi_smem = smem + C::kStages * C::kStageBytes;
     Ctl *ctl = reinterpret_cast<Ctl *>(epi_smem + C::kEpiBytes);
     constexpr int kBufs = C::kEpiBufs;      // staging tiles per group in the FP16-output path
+    constexpr int kPhases = C::kPhases, kEpiWarps = C::kEpiWarps, kStoreWarp0 = C::kStoreWarp0, kI8Bufs = C::kI8Bufs;
     volatile uint32_t *abort_flag = &ctl->abort_flag;
 
     const int warp = threadIdx.x >> 5;
@@ -641,11 +652,10 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             ptx::mbar_init(ptx::smem_u32(&ctl->tmem_empty[a]), 2 * kEpiWarps);   // the epilogue warps of both CTAs
         }
         ptx::mbar_init(ptx::smem_u32(&ctl->drain), 1);
-        for (int g = 0; g < kEpiGroups; ++g)
-            for (int b = 0; b < gpusq::kEpiBufs; ++b) {
-                ptx::mbar_init(ptx::smem_u32(&ctl->stg_full[g][b]), kOut == GPUSQ_OUT_I8 ? 8 : 4);
-                ptx::mbar_init(ptx::smem_u32(&ctl->stg_free[g][b]), 1);
-            }
+        for (int g = 0; g < C::kEpiGroups * kBufs; ++g) {
+            ptx::mbar_init(ptx::smem_u32(&ctl->stg_full[g]), kOut == GPUSQ_OUT_I8 ? 8 : 4);
+            ptx::mbar_init(ptx::smem_u32(&ctl->stg_free[g]), 1);
+        }
         ctl->abort_flag = 0;
         ctl->wait_us = p.wait_us;
         ptx::fence_barrier_init();
@@ -829,7 +839,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // tiles back to the epilogue warps once the stores have read them.
         if (kOut == GPUSQ_OUT_F16 && ptx::elect_one()) {
             const int fgroup = warp - kStoreWarp0;         // features [64 fgroup, 64 fgroup + 64) of the CTA's 128
-            uint32_t filled0 = 0, filled1 = 0;             // staging tiles stored so far, per chunk parity group
+            uint32_t filled[kMaxPhases] = {};              // staging tiles stored so far, per chunk phase
             uint32_t prev1 = 0, prev2 = 0;                 // free barriers of the last two stores (0 = none)
             int local = 0;
             bool ok = true;
@@ -843,12 +853,12 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 const int64_t left = p.M - m0;
                 const int nchunks = left >= h ? h / kChunkT : (int)((left + kChunkT - 1) / kChunkT);
                 for (int c = 0; c < nchunks; ++c) {
-                    const int par = (c + local) & 1;       // the group of warps that fills this chunk
-                    const int gi = fgroup * 2 + par;
-                    const uint32_t count = par ? filled1 : filled0;
+                    const int par = (c + kPhases - local % kPhases) % kPhases;     // the warps with (par + local) % kPhases == c % kPhases fill this chunk
+                    const int gi = fgroup * kPhases + par;
+                    const uint32_t count = filled[par];
                     const uint32_t b = count % kBufs;
                     bool to;
-                    if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->stg_full[gi][b]), (count / kBufs) & 1u,
+                    if (!ptx::mbar_wait_bounded(ptx::smem_u32(&ctl->stg_full[gi * kBufs + (int)b]), (count / kBufs) & 1u,
                                                 abort_flag, to)) {
                         if (to) report_timeout(p, ctl, tile, 3, gi * 8 + (int)b);
                         ok = false;
@@ -861,21 +871,19 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     ptx::tma_store_wait_read<2>();
                     if (prev2) ptx::mbar_arrive(prev2);
                     prev2 = prev1;
-                    prev1 = ptx::smem_u32(&ctl->stg_free[gi][b]);
-                    if (par) ++filled1; else ++filled0;
+                    prev1 = ptx::smem_u32(&ctl->stg_free[gi * kBufs + (int)b]);
+                    ++filled[par];
                 }
             }
             // the staging tiles must stay valid until the bulk stores have read them, and the
             // stores must be complete before the kernel ends
             ptx::tma_store_wait_all<0>();
         } else if (kOut == GPUSQ_OUT_I8 && ptx::elect_one()) {
-            // INT8 output: a staging tile holds all 128 features of a chunk; this lane serves the ring of
-            // one chunk parity (the parity groups swap every tile)
-            const int ring = warp - kStoreWarp0;
-            const uint8_t *ring_smem = epi_smem + ring * kI8Bufs * kEpiBufBytes;
-            const uint32_t full0 = ptx::smem_u32(&ctl->stg_full[0][0]) + (uint32_t)(ring * kI8Bufs * 8);
-            const uint32_t free0 = ptx::smem_u32(&ctl->stg_free[0][0]) + (uint32_t)(ring * kI8Bufs * 8);
-            uint32_t filled = 0;                           // staging tiles stored so far
+            // INT8 output: a staging tile holds all 128 features of a chunk; every chunk phase has its
+            // ring; this lane serves the rings of even (first store warp) or odd phases
+            const int odd = warp - kStoreWarp0;
+            const uint32_t full0 = ptx::smem_u32(&ctl->stg_full[0]), free0 = ptx::smem_u32(&ctl->stg_free[0]);
+            uint32_t filled[kMaxPhases] = {};              // staging tiles stored so far, per ring
             uint32_t prev1 = 0, prev2 = 0;
             int local = 0;
             bool ok = true;
@@ -888,22 +896,25 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 if (n0 >= p.N) continue;
                 const int64_t left = p.M - m0;
                 const int nchunks = left >= h ? h / kChunkT : (int)((left + kChunkT - 1) / kChunkT);
-                for (int c = (ring + local) & 1; c < nchunks; c += 2) {
-                    const uint32_t b = filled % kI8Bufs;
+                for (int c = 0; c < nchunks; ++c) {
+                    const int ring = (c + kPhases - local % kPhases) % kPhases;
+                    if ((ring & 1) != odd) continue;
+                    const uint32_t count = filled[ring];
+                    const uint32_t slot = (uint32_t)(ring * kI8Bufs) + count % kI8Bufs;
                     bool to;
-                    if (!ptx::mbar_wait_bounded(full0 + 8u * b, (filled / kI8Bufs) & 1u, abort_flag, to)) {
-                        if (to) report_timeout(p, ctl, tile, 3, ring * 8 + (int)b);
+                    if (!ptx::mbar_wait_bounded(full0 + 8u * slot, (count / kI8Bufs) & 1u, abort_flag, to)) {
+                        if (to) report_timeout(p, ctl, tile, 3, (int)slot);
                         ok = false;
                         break;
                     }
-                    ptx::tma_store_2d(&map_y, ptx::smem_u32(ring_smem + (int)b * kEpiBufBytes), n0,
+                    ptx::tma_store_2d(&map_y, ptx::smem_u32(epi_smem + (int)slot * kEpiBufBytes), n0,
                                       (int32_t)(m0 + c * kChunkT));
                     ptx::tma_store_commit();
                     ptx::tma_store_wait_read<2>();
                     if (prev2) ptx::mbar_arrive(prev2);
                     prev2 = prev1;
-                    prev1 = free0 + 8u * b;
-                    ++filled;
+                    prev1 = free0 + 8u * slot;
+                    ++filled[ring];
                 }
             }
             ptx::tma_store_wait_all<0>();
@@ -917,18 +928,18 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         // the accumulators of both CTAs are released on CTA 0's barrier, where the MMA issuer waits
         const uint32_t tmem_empty0 = ptx::map_to_cta(ptx::smem_u32(&ctl->tmem_empty[0]), 0);
         const uint32_t tmem_empty1 = ptx::map_to_cta(ptx::smem_u32(&ctl->tmem_empty[1]), 0);
-        const int group = (quarter >> 1) * 2 + par;        // 64 features x chunk parity: the warps sharing staging tiles
+        const int group = (quarter >> 1) * kPhases + par;  // 64 features x chunk phase: the warps sharing staging tiles
         const uint32_t stage0 = ptx::smem_u32(epi_smem + group * kBufs * kEpiBufBytes);
         int local = 0;
 
         if (kOut == GPUSQ_OUT_F16) {
-            EpiF16<kHalf, kBufs, kTwin> e;
+            EpiF16<kHalf, kBufs, kPhases, kTwin> e;
             e.p = &p;
             e.ctl = ctl;
             e.tmem_base = tmem_base;
             e.stage0 = stage0;
-            e.stg_full0 = ptx::smem_u32(&ctl->stg_full[group][0]);
-            e.stg_free0 = ptx::smem_u32(&ctl->stg_free[group][0]);
+            e.stg_full0 = ptx::smem_u32(&ctl->stg_full[group * kBufs]);
+            e.stg_free0 = ptx::smem_u32(&ctl->stg_free[group * kBufs]);
             e.tmem_empty0 = tmem_empty0;
             e.tmem_empty1 = tmem_empty1;
             e.x_scale = x_scale;
@@ -944,7 +955,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             else
                 e.template run<false, kAmax>();
         } else if (kOut == GPUSQ_OUT_I8) {
-            EpiI8<kTwin> e;
+            EpiI8<kI8Bufs, kPhases, kTwin> e;
             e.p = &p;
             e.ctl = ctl;
             e.epi_smem = epi_smem;
@@ -1209,7 +1220,7 @@ static int max_clusters(int sms)
     if (cached[dev] == 0) {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)(sms & ~1), 1, 1);
-        cfg.blockDim = dim3(kNumThreads, 1, 1);
+        cfg.blockDim = dim3(Cfg<kSparse, kHalf>::kThreads, 1, 1);
         cfg.dynamicSmemBytes = Cfg<kSparse, kHalf>::kSmemBytes;
         int n = 0;
         if (cudaOccupancyMaxActiveClusters(&n, gemm_i8_kernel<kSparse, GPUSQ_OUT_F16, kHalf>, &cfg) != cudaSuccess || n <= 0) {
@@ -1267,14 +1278,14 @@ static bool prepare_device(int kind)
 }
 
 template <typename Kernel>
-static int launch_on(Kernel kernel, int smem_bytes, const CUtensorMap &map_a, const CUtensorMap &map_b,
+static int launch_on(Kernel kernel, int threads, int smem_bytes, const CUtensorMap &map_a, const CUtensorMap &map_b,
                      const CUtensorMap &map_b2, const CUtensorMap &map_e, const CUtensorMap &map_y,
                      const GemmParams &p, int clusters, void *stream)
 {
     const int grid = 2 * (p.num_tiles < clusters ? p.num_tiles : clusters);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid, 1, 1);
-    cfg.blockDim = dim3(kNumThreads, 1, 1);
+    cfg.blockDim = dim3((unsigned)threads, 1, 1);
     cfg.dynamicSmemBytes = smem_bytes;
     cfg.stream = (cudaStream_t)stream;
     cudaLaunchAttribute attr[1];
@@ -1357,16 +1368,16 @@ static int launch_gemm(const int8_t *Xq, const void *Wsrc, const float *w_scale,
     // launches without a twin column run the instantiation that has no trace of it
     const int smem = C::kSmemBytes;
     if (out_type == GPUSQ_OUT_F16 && y_absmax && kSparse)
-        return twin_col ? launch_on(gemm_i8_kernel<true, GPUSQ_OUT_F16, false, true, true>, smem, map_a, map_b, map_b2, map_e, map_y, p, clusters, stream)
-                        : launch_on(gemm_i8_kernel<true, GPUSQ_OUT_F16, false, false, true>, smem, map_a, map_b, map_b2, map_e, map_y, p, clusters, stream);
+        return twin_col ? launch_on(gemm_i8_kernel<true, GPUSQ_OUT_F16, false, true, true>, C::kThreads, smem, map_a, map_b, map_b2, map_e, map_y, p, clusters, stream)
+                        : launch_on(gemm_i8_kernel<true, GPUSQ_OUT_F16, false, false, true>, C::kThreads, smem, map_a, map_b, map_b2, map_e, map_y, p, clusters, stream);
     if (out_type == GPUSQ_OUT_F16)
-        return twin_col ? launch_on(gemm_i8_kernel<kSparse, GPUSQ_OUT_F16, false, true>, smem, map_a, map_b, map_b2, map_e, map_y, p, clusters, stream)
-                        : launch_on(gemm_i8_kernel<kSparse, GPUSQ_OUT_F16>, smem, map_a, map_b, map_b2, map_e, map_y, p, clusters, stream);
+        return twin_col ? launch_on(gemm_i8_kernel<kSparse, GPUSQ_OUT_F16, false, true>, C::kThreads, smem, map_a, map_b, map_b2, map_e, map_y, p, clusters, stream)
+                        : launch_on(gemm_i8_kernel<kSparse, GPUSQ_OUT_F16>, C::kThreads, smem, map_a, map_b, map_b2, map_e, map_y, p, clusters, stream);
     if (out_type == GPUSQ_OUT_I8)
-        return twin_col ? launch_on(gemm_i8_kernel<kSparse, GPUSQ_OUT_I8, false, true>, smem, map_a, map_b, map_b2, map_e, map_y, p, clusters, stream)
-                        : launch_on(gemm_i8_kernel<kSparse, GPUSQ_OUT_I8>, smem, map_a, map_b, map_b2, map_e, map_y, p, clusters, stream);
-    return twin_col ? launch_on(gemm_i8_kernel<kSparse, GPUSQ_OUT_I32, false, true>, smem, map_a, map_b, map_b2, map_e, map_y, p, clusters, stream)
-                    : launch_on(gemm_i8_kernel<kSparse, GPUSQ_OUT_I32>, smem, map_a, map_b, map_b2, map_e, map_y, p, clusters, stream);
+        return twin_col ? launch_on(gemm_i8_kernel<kSparse, GPUSQ_OUT_I8, false, true>, C::kThreads, smem, map_a, map_b, map_b2, map_e, map_y, p, clusters, stream)
+                        : launch_on(gemm_i8_kernel<kSparse, GPUSQ_OUT_I8>, C::kThreads, smem, map_a, map_b, map_b2, map_e, map_y, p, clusters, stream);
+    return twin_col ? launch_on(gemm_i8_kernel<kSparse, GPUSQ_OUT_I32, false, true>, C::kThreads, smem, map_a, map_b, map_b2, map_e, map_y, p, clusters, stream)
+                    : launch_on(gemm_i8_kernel<kSparse, GPUSQ_OUT_I32>, C::kThreads, smem, map_a, map_b, map_b2, map_e, map_y, p, clusters, stream);
 }
 
 // The FP16 2:4 sparse layer: binary16 activations as they are, FP32 accumulation, bias, optional GELU.
@@ -1423,10 +1434,10 @@ static int launch_gemm_f16(const void *X, const void *Wpacked, const float *bias
 
     const int smem = C::kSmemBytes;
     if (out_type == GPUSQ_OUT_F16)
-        return twin_col ? launch_on(gemm_i8_kernel<true, GPUSQ_OUT_F16, true, true>, smem, map_a, map_b, map_b2, map_e, map_y, p, clusters, stream)
-                        : launch_on(gemm_i8_kernel<true, GPUSQ_OUT_F16, true>, smem, map_a, map_b, map_b2, map_e, map_y, p, clusters, stream);
-    return twin_col ? launch_on(gemm_i8_kernel<true, GPUSQ_OUT_I32, true, true>, smem, map_a, map_b, map_b2, map_e, map_y, p, clusters, stream)
-                    : launch_on(gemm_i8_kernel<true, GPUSQ_OUT_I32, true>, smem, map_a, map_b, map_b2, map_e, map_y, p, clusters, stream);
+        return twin_col ? launch_on(gemm_i8_kernel<true, GPUSQ_OUT_F16, true, true>, C::kThreads, smem, map_a, map_b, map_b2, map_e, map_y, p, clusters, stream)
+                        : launch_on(gemm_i8_kernel<true, GPUSQ_OUT_F16, true>, C::kThreads, smem, map_a, map_b, map_b2, map_e, map_y, p, clusters, stream);
+    return twin_col ? launch_on(gemm_i8_kernel<true, GPUSQ_OUT_I32, true, true>, C::kThreads, smem, map_a, map_b, map_b2, map_e, map_y, p, clusters, stream)
+                    : launch_on(gemm_i8_kernel<true, GPUSQ_OUT_I32, true>, C::kThreads, smem, map_a, map_b, map_b2, map_e, map_y, p, clusters, stream);
 }
 
 }  // namespace gpusq
