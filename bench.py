@@ -14,6 +14,7 @@ host cores instead (a deliberately plain program: context, not a target).
 from __future__ import annotations
 
 import argparse
+import collections
 import json
 import math
 import os
@@ -852,6 +853,100 @@ def run_patch_embed(args, pcfg):
     print(json.dumps(line))
 
 
+# ------------------------------------------------------------------- time per tile of a few CTA pairs
+def run_tile_sweep(args, cfg):
+    """Time per output tile of one CTA pair, with and without the other SMs' traffic.
+
+    The GEMM launches are held to `pairs` CTA pairs (measurement hook of gpusq_testing.h) and the
+    tokens are cut so that every pair works on 8 and then on 16 tiles of 224 tokens: the difference
+    is eight tile periods in steady state, the rest the launch's fixed cost.  `pairs` = 9 leaves
+    130 of 148 SMs idle (what one pair can do by itself); `pairs` = all is the loaded GPU.  One JSON
+    line; single GPU; not a throughput figure.
+    """
+    import torch
+
+    from paper_2305_10727_b200 import binding as B
+
+    if int(os.environ.get("WORLD_SIZE", "1")) != 1:
+        raise SystemExit("--tile-sweep is a single-GPU measurement")
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: libgpusq has no CPU fallback")
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    B.load()
+    stream = torch.cuda.Stream()
+    torch.cuda.set_stream(stream)
+    block_t = 224
+    B.set_block_tokens(block_t)
+    sm_mhz = None
+
+    def timed_us(fn, nbuf):
+        for i in range(nbuf):
+            fn(i)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for i in range(nbuf):
+                fn(i)
+        for _ in range(max(3, args.warmup)):
+            g.replay()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record(stream)
+        for _ in range(10):
+            g.replay()
+        b.record(stream)
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / (10 * nbuf) * 1e3
+
+    all_pairs = torch.cuda.get_device_properties(dev).multi_processor_count // 2
+    rows = []
+    sampler = ClockSampler(0)
+    sampler.start()
+    try:
+        # the layers of the block, and one shape whose main loop is two k blocks: the epilogue alone
+        short = collections.namedtuple("Shape", "name N K")("k256", cfg.layers[0].N, 256)
+        for L in list(cfg.layers) + [short]:
+            d = inputs.random_layer(1000 + L.N + L.K, 64, L.N, L.K)
+            Wq, ws = B.quant_weight(B.prune24(torch.from_numpy(d["W"]).to(dev)))
+            Wpk = B.pack24(*B.compress24(Wq))
+            bias = torch.from_numpy(d["bias"]).to(dev)
+            cols = (L.N + 255) // 256
+            xs = torch.tensor([0.01], dtype=torch.float32, device=dev)
+            osc = torch.tensor([0.05], dtype=torch.float32, device=dev)
+            status = torch.zeros(4, dtype=torch.int32, device=dev)
+            for kind, act, ot in (("f16", 0, B.OUT_F16), ("f16+gelu", 1, B.OUT_F16), ("i8", 0, B.OUT_I8)):
+                for pairs in (9, all_pairs):
+                    B.set_max_clusters(pairs)
+                    t = []
+                    for per_pair in (8, 16):
+                        # tiles = cols x token tiles = pairs x per_pair
+                        tok_tiles = max(1, (pairs * per_pair) // cols)
+                        M = tok_tiles * block_t
+                        Xq = torch.randint(-127, 128, (M, L.K), dtype=torch.int8, device=dev)
+                        odt = torch.float16 if ot == B.OUT_F16 else torch.int8
+                        Y = [torch.empty((M, L.N), dtype=odt, device=dev) for _ in range(4)]
+                        t.append((timed_us(lambda i: B.spgemm_i8(Xq, Wpk, L.N, ws, xs, bias, act=act, out_type=ot,
+                                                                  out_scale=osc, Y=Y[i], status_buf=status), 4),
+                                  -(-(cols * tok_tiles) // pairs)))
+                    per_tile = (t[1][0] - t[0][0]) / (t[1][1] - t[0][1])
+                    rows.append({"layer": L.name, "N": L.N, "K": L.K, "out": kind, "pairs": pairs,
+                                 "us_8_tiles": round(t[0][0], 2), "us_16_tiles": round(t[1][0], 2),
+                                 "tiles_per_pair": [t[0][1], t[1][1]],
+                                 "us_per_tile": round(per_tile, 3), "fixed_us": round(t[0][0] - per_tile * t[0][1], 2)})
+            if status.cpu().tolist() != [0, 0, 0, 0]:
+                raise SystemExit("device status %s" % status.cpu().tolist())
+    finally:
+        B.set_max_clusters(0)
+        B.set_block_tokens(0)
+        clocks = sampler.stop()
+    for r in rows:
+        if clocks.get("sm_mhz"):
+            r["cycles_per_tile"] = int(round(r["us_per_tile"] * clocks["sm_mhz"]))
+    print(json.dumps({"tile_sweep": rows, "block_tokens": block_t, "config": {"workload": args.config},
+                      "clocks": clocks, "note": "time per 256-feature x 224-token tile of one CTA pair: (t(16 tiles) - t(8 tiles)) / 8"}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -866,10 +961,15 @@ def main():
                     help="token rows per layer the CPU oracle is timed on with all host cores (a quarter of them on one core)")
     ap.add_argument("--ref-rows-reference", type=int, default=0,
                     help="token rows per step for --impl reference (0 = size from a calibration run)")
+    ap.add_argument("--tile-sweep", action="store_true",
+                    help="time per output tile of one CTA pair on 9 pairs and on all of them (measurement aid, not a throughput figure)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     cfg = inputs.CONFIGS[args.config]
+    if args.tile_sweep and args.impl == "gpusq":
+        run_tile_sweep(args, cfg)
+        return
     if args.patch is not None and args.impl == "gpusq":
         run_patch_embed(args, inputs.PATCH_CONFIGS[args.patch])
         return

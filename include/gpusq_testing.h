@@ -3,7 +3,8 @@
  * program that uses libgpusq.so has no reason to call these (the paper has no
  * counterpart).  They exist so that the parity tests can drive the GEMM
  * kernels through every tile height and through mixed tile heights on small
- * shapes; results never depend on them.
+ * shapes, and so that the measurement script can time a few CTA pairs alone;
+ * results never depend on them.
  *
  * All settings are process-wide atomics read by every later call of the
  * process, from any thread; they are meant to be set while no other thread is
@@ -40,6 +41,12 @@ int gpusq_set_quant_act_wait(unsigned long long limit_ns, int withhold_last_cta)
  * stage} to status_buf, every role of the pair leaves its loop, and the kernel
  * returns.  The other pairs finish their tiles.  Nothing faults or hangs. */
 int gpusq_set_gemm_wait(unsigned limit_us, int withhold_loads);
+
+/* Measurement hook: the GEMM launches use at most `clusters` CTA pairs (0 = as
+ * many as the GPU holds, the default).  With the tokens cut in proportion,
+ * every pair keeps its number of tiles, so the time per tile of one pair can
+ * be read with little or no traffic from the other SMs (bench.py --tile-sweep). */
+int gpusq_set_max_clusters(int clusters);
 
 #ifdef __cplusplus
 }

@@ -24,7 +24,7 @@ SCALE_COMPUTE, SCALE_GIVEN = 0, 1
 EXPORTS = (
     "gpusq_status_string", "gpusq_prune24", "gpusq_quant_weight", "gpusq_compress24",
     "gpusq_decompress24", "gpusq_packed_bytes", "gpusq_pack24", "gpusq_quant_act_workspace",
-    "gpusq_quant_act", "gpusq_quant_act_static", "gpusq_patch_quant", "gpusq_spgemm_i8", "gpusq_gemm_i8_dense", "gpusq_set_block_tokens", "gpusq_set_tile_mix", "gpusq_set_quant_act_wait", "gpusq_set_gemm_wait",
+    "gpusq_quant_act", "gpusq_quant_act_static", "gpusq_patch_quant", "gpusq_spgemm_i8", "gpusq_gemm_i8_dense", "gpusq_set_block_tokens", "gpusq_set_tile_mix", "gpusq_set_quant_act_wait", "gpusq_set_gemm_wait", "gpusq_set_max_clusters",
     "gpusq_spgemm_i8_absmax", "gpusq_quant_act_absmax",
     "gpusq_prune48", "gpusq_quant_weight4", "gpusq_compress48", "gpusq_expand48", "gpusq_quant_act4",
     "gpusq_compress24_f16", "gpusq_packed_bytes_f16", "gpusq_pack24_f16", "gpusq_spgemm_f16",
@@ -78,6 +78,7 @@ def load() -> ctypes.CDLL:
     lib.gpusq_set_tile_mix.argtypes = [i32, i32]
     lib.gpusq_set_quant_act_wait.argtypes = [ctypes.c_ulonglong, i32]
     lib.gpusq_set_gemm_wait.argtypes = [ctypes.c_uint, i32]
+    lib.gpusq_set_max_clusters.argtypes = [i32]
     lib.gpusq_compress24_f16.argtypes = [vp, vp, vp, i32, i32, vp]
     lib.gpusq_packed_bytes_f16.argtypes = [i32, i32]
     lib.gpusq_packed_bytes_f16.restype = sz
@@ -322,6 +323,11 @@ def gemm_i8_dense(Xq: torch.Tensor, Wq: torch.Tensor, w_scale=None, x_scale=None
 def set_block_tokens(block_t: int) -> None:
     """Test hook (gpusq_testing.h): force the GEMM tile height; 0 = automatic."""
     _check(load().gpusq_set_block_tokens(block_t), "gpusq_set_block_tokens")
+
+
+def set_max_clusters(clusters: int) -> None:
+    """Measurement hook (gpusq_testing.h): the GEMM launches use at most that many CTA pairs (0 = all)."""
+    _check(load().gpusq_set_max_clusters(int(clusters)), "gpusq_set_max_clusters")
 
 
 def set_tile_mix(block_t: int, n_big: int) -> None:

@@ -1076,6 +1076,7 @@ static std::atomic<int> g_block_t_override{0};
 static std::atomic<int> g_n_big_override{-1};
 static std::atomic<unsigned> g_wait_us{ptx::kDefaultWaitUs};
 static std::atomic<int> g_withhold_loads{0};
+static std::atomic<int> g_cluster_cap{0};           // CTA pairs a launch may use (0 = as many as fit)
 
 // How the token axis is cut into tiles: tok_tiles token tiles, the first n_big of them block_t tokens
 // high, the others block_t - 32.
@@ -1232,6 +1233,13 @@ static int max_clusters(int sms)
     return cached[dev];
 }
 
+// measurement hook (gpusq_testing.h): fewer CTA pairs than fit
+static int capped(int clusters)
+{
+    const int cap = g_cluster_cap.load(std::memory_order_relaxed);
+    return cap > 0 && cap < clusters ? cap : clusters;
+}
+
 // The kernels need more dynamic shared memory than the default limit; the attribute is per device.
 template <typename F>
 static bool allow_smem(F kernel, int bytes)
@@ -1318,7 +1326,7 @@ static int launch_gemm(const int8_t *Xq, const void *Wsrc, const float *w_scale,
     if (!prepare_device(kSparse ? 0 : 1)) return GPUSQ_ERR_CUDA;
 
     const int sms = num_sms();
-    const int clusters = max_clusters<kSparse>(sms);
+    const int clusters = capped(max_clusters<kSparse>(sms));
     if (clusters <= 0) return GPUSQ_ERR_CUDA;
 
     GemmParams p;
@@ -1394,7 +1402,7 @@ static int launch_gemm_f16(const void *X, const void *Wpacked, const float *bias
     if (!prepare_device(2)) return GPUSQ_ERR_CUDA;
 
     const int sms = num_sms();
-    const int clusters = max_clusters<true, true>(sms);
+    const int clusters = capped(max_clusters<true, true>(sms));
     if (clusters <= 0) return GPUSQ_ERR_CUDA;
 
     GemmParams p;
@@ -1493,6 +1501,13 @@ int gpusq_set_gemm_wait(unsigned limit_us, int withhold_loads)
     if (limit_us == 0) return GPUSQ_ERR_ARG;
     g_wait_us.store(limit_us, std::memory_order_relaxed);
     g_withhold_loads.store(withhold_loads ? 1 : 0, std::memory_order_relaxed);
+    return GPUSQ_OK;
+}
+
+int gpusq_set_max_clusters(int clusters)
+{
+    if (clusters < 0) return GPUSQ_ERR_ARG;
+    g_cluster_cap.store(clusters, std::memory_order_relaxed);
     return GPUSQ_OK;
 }
 
