@@ -224,6 +224,28 @@ def test_mixed_tile_heights(B, M, N, K, block_t, n_big):
     assert np.array_equal(Q, Q_o)
 
 
+@pytest.mark.parametrize("pairs", [1, 3, 20])
+def test_fewer_cta_pairs_same_result(B, pairs):
+    # the measurement hook that holds a launch to a few CTA pairs changes who computes a tile, never the tile:
+    # accumulators and FP16 + GELU output against the oracle, with many tiles per pair and a ragged end
+    M, N, K = 1576, 768, 192
+    d, prep, Xq, xs = _prep(5 * M + N + K + pairs, M, N, K)
+    acc_o = oracle.spgemm_acc(Xq, prep["vals"], prep["meta"], threads=oracle.host_cores())
+    Y_o = oracle.epilogue(acc_o, prep["w_scale"], xs, d["bias"], act=1, out_type=0, threads=oracle.host_cores())
+    Wpk = B.pack24(cu(prep["vals"]), cu(prep["meta"]))
+    status = torch.zeros(4, dtype=torch.int32, device="cuda")
+    B.set_max_clusters(pairs)
+    try:
+        acc = B.spgemm_i8(cu(Xq), Wpk, N, out_type=B.OUT_I32, status_buf=status).cpu().numpy()
+        Y = B.spgemm_i8(cu(Xq), Wpk, N, cu(prep["w_scale"]), cu(np.array([xs], np.float32)), cu(d["bias"]),
+                        act=B.ACT_GELU, out_type=B.OUT_F16, status_buf=status).cpu().numpy()
+    finally:
+        B.set_max_clusters(0)
+    assert status.cpu().tolist() == [0, 0, 0, 0]
+    assert np.array_equal(acc, acc_o)
+    assert f16_ulp_distance(Y, Y_o).max() <= F16_ULP_TOL
+
+
 def test_gemm_wait_that_runs_out_is_reported(B):
     # A planted failure in an allowed form: the first CTA pair's loads for the last k block of its first tile
     # are never issued, so the MMA issuer's bounded wait (5 ms here) runs out.  Expected: status_buf =
